@@ -1,0 +1,461 @@
+"""Pins for the CPU oracle: closed forms, exact rational brute force, invariants and
+special cases that reduce to library routines.  None of these restate the oracle's
+own code path; a dropped term, wrong sign, off-by-one or transposed operand in the
+oracle fails at least one of them."""
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import Params
+
+RNG = np.random.default_rng(20260523)
+
+
+# ----------------------------------------------------------------------------- Eq. 1
+
+def test_mass_eq1_closed_form_dyadic():
+    # weights that are exact in fp32 and in 36-bit fixed point: the mass is the exact ratio
+    eps = 2.0 ** -10
+    u = np.array([1.0, 3.0, -5.0, 0.0, 4.0 - eps, float("nan")], dtype=np.float32)
+    A, SA, m = oracle.mass(u, eps)
+    w = [Fraction(1) + Fraction(eps), Fraction(3) + Fraction(eps), Fraction(eps), Fraction(eps), Fraction(4),
+         Fraction(eps)]
+    tot = sum(w)
+    for t in range(len(u)):
+        assert Fraction(int(A[t]), SA) == w[t] / tot            # fixed point kept the ratios exactly
+        assert m[t] == np.float32(float(w[t] / tot))            # one rounding to fp32
+    assert int(A.sum()) == SA
+
+
+def test_mass_sums_to_one_and_floor():
+    for T in (1, 7, 4096, 131072):
+        u = RNG.standard_normal(T).astype(np.float32)
+        A, SA, m = oracle.mass(u, 1e-8)
+        assert abs(float(m.astype(np.float64).sum()) - 1.0) <= T * 2.0 ** -24
+        assert (m > 0).all() or (A == 0).any()
+        assert int(A.max()) >= 2 ** 35 and int(A.max()) < 2 ** 36
+        # negative scores carry only epsilon: all equal, and the smallest
+        neg = u <= 0
+        if neg.any():
+            assert len(np.unique(m[neg])) == 1 and m[neg][0] == m.min()
+
+
+def test_mass_scale_invariance_power_of_two():
+    u = np.abs(RNG.standard_normal(257)).astype(np.float32) + 0.5
+    A1, S1, m1 = oracle.mass(u, 0.0 + 2.0 ** -40)
+    A2, S2, m2 = oracle.mass(u * np.float32(1024.0), 2.0 ** -30)
+    assert (A1 == A2).all() and S1 == S2 and (m1 == m2).all()
+
+
+# ----------------------------------------------------------------------------- cuts
+
+def _brute_cuts(w, S):
+    """Exact rational statement: b_k = min{t : c(t) >= k/S} with 1-based t, k = 1..S-1."""
+    T = len(w)
+    tot = sum(w)
+    out = {0, T}
+    for k in range(1, S):
+        c = Fraction(0)
+        for t in range(1, T + 1):
+            c += w[t - 1]
+            if c / tot >= Fraction(k, S):
+                if 0 < t < T:
+                    out.add(t)
+                break
+    return sorted(out)
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_cuts_match_exact_rational_brute_force(seed):
+    rng = np.random.default_rng(seed)
+    T = int(rng.integers(2, 65))
+    S = int(rng.integers(1, 13))
+    # small integer scores; eps = 2^-12 keeps every weight exact in fp32 and in fixed point
+    eps = 2.0 ** -12
+    u = rng.integers(-3, 40, size=T).astype(np.float32)
+    if seed % 5 == 0:
+        u[int(rng.integers(0, T))] = 4000.0          # one spike crossing several thresholds
+    w = [Fraction(max(float(x), 0.0)) + Fraction(eps) for x in u]
+    A, SA, m = oracle.mass(u, eps)
+    Hm, _ = oracle.history_mass(A, SA, m, np.zeros(T, np.float32), 0.9, 1.0)
+    got = oracle.cuts(oracle.prefix(Hm), S)
+    assert got.tolist() == _brute_cuts(w, S)
+
+
+def test_cuts_uniform_mass_closed_form():
+    for T, S in ((100, 10), (4096, 8), (60, 3), (64, 64)):
+        u = np.full(T, 0.25, dtype=np.float32)
+        A, SA, m = oracle.mass(u, 1e-8)
+        Hm, _ = oracle.history_mass(A, SA, m, np.zeros(T, np.float32), 0.9, 1.0)
+        b = oracle.cuts(oracle.prefix(Hm), S)
+        assert b.tolist() == [k * (T // S) for k in range(S + 1)]
+
+
+def test_cuts_spike_dedup_and_single_segment():
+    T = 50
+    u = np.full(T, 1e-3, dtype=np.float32)
+    u[20] = 100.0                                      # holds > 99.9 % of the mass
+    A, SA, m = oracle.mass(u, 1e-8)
+    Hm, _ = oracle.history_mass(A, SA, m, np.zeros(T, np.float32), 0.9, 1.0)
+    C = oracle.prefix(Hm)
+    assert oracle.cuts(C, 10).tolist() == [0, 21, T]   # one cut right after the spike, no empty segments
+    assert oracle.cuts(C, 1).tolist() == [0, T]
+    u[:] = 1e-3
+    u[T - 1] = 100.0                                   # spike on the last token: its cut would be T, dropped
+    A, SA, m = oracle.mass(u, 1e-8)
+    Hm, _ = oracle.history_mass(A, SA, m, np.zeros(T, np.float32), 0.9, 1.0)
+    assert oracle.cuts(oracle.prefix(Hm), 4).tolist() == [0, T]
+
+
+# ----------------------------------------------------------------------------- merge / split
+
+@pytest.mark.parametrize("seed", range(60))
+def test_merge_split_invariants(seed):
+    rng = np.random.default_rng(1000 + seed)
+    T = int(rng.integers(1, 3000))
+    n_cut = int(rng.integers(0, 30))
+    raw = sorted({0, T} | {int(x) for x in rng.integers(1, max(T, 2), size=n_cut) if 0 < x < T})
+    l_min = int(rng.integers(1, 40))
+    l_max = int(rng.choice([0, 2 * l_min, 2 * l_min + 7, 256, 1000]))
+    b = oracle.merge_split(np.array(raw, np.int32), l_min, l_max)
+    lens = np.diff(b)
+    assert b[0] == 0 and b[-1] == T and (lens > 0).all()             # cover, disjoint, ordered
+    if T >= l_min and (l_max == 0 or l_max >= 2 * l_min):
+        assert (lens >= l_min).all()
+    if l_max > 0:
+        assert (lens <= l_max).all()
+    if l_max == 0:
+        assert set(b.tolist()) <= set(raw)                            # merging only removes boundaries
+    # every boundary that survives merging is a raw boundary; split pieces are near-equal
+    merged = [x for x in b.tolist() if x in set(raw)]
+    for a, e in zip(merged[:-1], merged[1:]):
+        inner = [x for x in b.tolist() if a <= x <= e]
+        pl = np.diff(inner)
+        assert pl.max() - pl.min() <= 1
+        assert list(pl) == sorted(pl, reverse=True)                   # larger pieces first
+        if l_max > 0:
+            assert len(pl) == -(-(e - a) // l_max) or (e - a) <= l_max
+
+
+def test_merge_split_examples():
+    # forward absorb: 5+5+10 -> 20 when l_min = 16; tail 4 folds left
+    assert oracle.merge_split(np.array([0, 5, 10, 20, 40, 44], np.int32), 16, 0).tolist() == [0, 20, 44]
+    # a single short segment stays
+    assert oracle.merge_split(np.array([0, 7], np.int32), 16, 256).tolist() == [0, 7]
+    # split 1000 with l_max 256 -> 4 pieces of 250
+    assert oracle.merge_split(np.array([0, 1000], np.int32), 16, 256).tolist() == [0, 250, 500, 750, 1000]
+    # 10 into l_max 4 -> ceil(10/4)=3 pieces 4,3,3
+    assert oracle.merge_split(np.array([0, 10], np.int32), 1, 4).tolist() == [0, 4, 7, 10]
+
+
+# ----------------------------------------------------------------------------- quotas
+
+def _prefix_from_masses(masses, lens):
+    """Cumulative integer mass with each segment's mass spread evenly over its tokens."""
+    Hm = np.concatenate([np.full(L, M // L, dtype=np.uint64) for M, L in zip(masses, lens)])
+    return np.cumsum(Hm, dtype=np.uint64)
+
+
+def test_quota_formula_worked_example():
+    # two long segments with masses 1:3, q_min = 1, budget 102: 1 + round(100/4) and 1 + round(300/4)
+    lens = [400, 400]
+    C = _prefix_from_masses([400 * 2 ** 20, 1200 * 2 ** 20], lens)
+    q = oracle.quotas(C, np.array([0, 400, 800], np.int32), 1, 102)
+    assert q.tolist() == [26, 76]
+    # clipping: shares 1+3, 1+91 -> clipped to 10, 1+6; the deficit of 82 is handed out one token
+    # per visit, heaviest segment with room first: 41 to each of the two long segments
+    lens = [300, 10, 300]
+    C = _prefix_from_masses([300 * 2 ** 20, 9000 * 2 ** 20, 600 * 2 ** 20], lens)
+    q = oracle.quotas(C, np.array([0, 300, 310, 610], np.int32), 1, 103)
+    assert q.tolist() == [45, 10, 48]
+    # budget below the minima: minima are given up lightest first (ties: higher index)
+    C = _prefix_from_masses([100 * 2 ** 20, 100 * 2 ** 20, 300 * 2 ** 20], [100, 100, 100])
+    assert oracle.quotas(C, np.array([0, 100, 200, 300], np.int32), 2, 4).tolist() == [1, 1, 2]
+    assert oracle.quotas(C, np.array([0, 100, 200, 300], np.int32), 2, 1).tolist() == [0, 0, 1]
+
+
+@pytest.mark.parametrize("seed", range(60))
+def test_quota_invariants(seed):
+    rng = np.random.default_rng(2000 + seed)
+    n_seg = int(rng.integers(1, 40))
+    lens = rng.integers(1, 300, size=n_seg)
+    masses = (rng.integers(1, 1000, size=n_seg).astype(np.int64) * lens) << 10
+    C = _prefix_from_masses(masses.tolist(), lens.tolist())
+    bounds = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    T = int(bounds[-1])
+    q_min = int(rng.integers(0, 5))
+    Bq = int(rng.integers(0, T + 1))
+    q = oracle.quotas(C, bounds, q_min, Bq)
+    qmin = np.minimum(q_min, lens)
+    assert q.sum() == Bq                                        # quotas sum to the budget
+    assert (q <= lens).all() and (q >= 0).all()
+    if qmin.sum() <= Bq:
+        assert (q >= qmin).all()                                 # minimum guarantee
+        # proportional share up to rounding and the greedy correction
+        M = np.diff(np.concatenate([[0], C[bounds[1:] - 1].astype(np.int64)]))
+        share = (Bq - qmin.sum()) * M / M.sum()
+        unclipped = q < lens
+        if unclipped.all():
+            assert np.abs(q - qmin - share).max() <= 1.5 + 1e-9
+
+
+def test_quota_equal_segments_equal_quotas():
+    lens = [100] * 8
+    C = _prefix_from_masses([100 * 2 ** 20] * 8, lens)
+    bounds = np.arange(0, 900, 100, dtype=np.int32)
+    q = oracle.quotas(C, bounds, 1, 84)        # 84 = 8*10 + 4: the first four (ties by index) get one more
+    assert q.tolist() == [11, 11, 11, 11, 10, 10, 10, 10]
+
+
+# ----------------------------------------------------------------------------- selection
+
+def _key_order(g):
+    """Library statement of the order: score descending, NaN last, ties by lower position."""
+    g = np.asarray(g, dtype=np.float32)
+    bits = g.view(np.uint32).astype(np.int64)
+    key = np.where(bits >> 31 == 1, (~bits) & 0xFFFFFFFF, bits | 0x80000000)
+    key = np.where(np.isnan(g), 0, key)
+    return np.lexsort((np.arange(len(g)), -key))
+
+
+@pytest.mark.parametrize("seed", range(20))
+def test_single_segment_is_global_topk(seed):
+    rng = np.random.default_rng(3000 + seed)
+    T = int(rng.integers(2, 5000))
+    Tk = int(rng.integers(1, T))
+    g = rng.standard_normal(T).astype(np.float32)
+    if seed % 3 == 0:
+        g = np.round(g * 2) / 2                         # many ties
+    if seed % 4 == 0:
+        g[rng.integers(0, T, size=3)] = np.nan
+        g[rng.integers(0, T, size=3)] = -0.0
+        g[rng.integers(0, T, size=3)] = np.inf
+    prm = Params(n_segments=1, l_min=1, l_max=0, q_min=0, n_sink=0, n_last=0, ema_beta=1.0)
+    res = oracle.select_unit(np.abs(g), g, None, Tk, prm)
+    assert res.n_seg == 1 and res.quotas.tolist() == [Tk] and res.n_backfill == 0
+    assert res.keep_idx.tolist() == sorted(_key_order(g)[:Tk].tolist())
+    # and against torch.topk on the values where no ties / NaN are involved
+    if seed % 3 != 0 and seed % 4 != 0:
+        assert set(res.keep_idx.tolist()) == set(torch.topk(torch.from_numpy(g), Tk).indices.tolist())
+
+
+@pytest.mark.parametrize("seed", range(30))
+def test_segmented_select_brute_force(seed):
+    rng = np.random.default_rng(4000 + seed)
+    T = int(rng.integers(8, 64))
+    n_seg = int(rng.integers(1, 6))
+    inner = sorted(set(rng.integers(1, T, size=n_seg - 1).tolist()))
+    bounds = np.array([0] + inner + [T], np.int32)
+    lens = np.diff(bounds)
+    q = np.array([int(rng.integers(0, L + 1)) for L in lens], np.int32)
+    g = rng.integers(-4, 5, size=T).astype(np.float32)           # heavy ties
+    ns, nl = int(rng.integers(0, 3)), int(rng.integers(0, 4))
+    chosen = set()
+    for i in range(len(q)):
+        a, b = int(bounds[i]), int(bounds[i + 1])
+        chosen |= set(sorted(range(a, b), key=lambda t: (-g[t], t))[:q[i]])
+    must = set(range(ns)) | set(range(T - nl, T))
+    union = chosen | must
+    Tk = int(q.sum()) + ns + nl
+    if Tk > T:
+        return
+    rest = sorted(set(range(T)) - union, key=lambda t: (-g[t], t))
+    want = sorted(union | set(rest[:Tk - len(union)]))
+    keep, r = oracle.select(g, bounds, q, ns, nl, Tk)
+    assert keep.tolist() == want and r == Tk - len(union)
+
+
+# ----------------------------------------------------------------------------- EMA
+
+def test_ema_closed_form_two_tokens():
+    eps = 2.0 ** -30
+    u = np.array([0.25, 0.75], np.float32)
+    A, SA, m = oracle.mass(u, eps)
+    Hm, c = oracle.history_mass(A, SA, m, np.array([0.5, 0.5], np.float32), 0.5, 0.5)
+    np.testing.assert_allclose(c, [0.375, 0.625], rtol=1e-6)
+    np.testing.assert_allclose(Hm.astype(np.float64) / 2 ** 36, [0.3125, 0.6875], rtol=1e-6)
+    # lambda = 0: the credit becomes the current mass
+    _, c0 = oracle.history_mass(A, SA, m, np.array([0.9, 0.1], np.float32), 0.0, 0.5)
+    assert (c0 == m).all()
+
+
+def test_ema_unit_beta_is_ema_off_and_first_event_is_neutral():
+    T, Tk = 1500, 400
+    u = np.abs(RNG.standard_normal(T)).astype(np.float32) ** 3
+    junk = RNG.random(T).astype(np.float32)
+    off = oracle.select_unit(u, u, junk, Tk, Params(ema_beta=1.0))
+    off2 = oracle.select_unit(u, u, None, Tk, Params(ema_beta=1.0, ema_lambda=0.3))
+    assert (off.credit == junk).all()                                     # credit untouched
+    assert off.bounds.tolist() == off2.bounds.tolist() and (off.keep_idx == off2.keep_idx).all()
+    # first event, zero credit: normalize(c) = m, so the mixed mass equals m up to rounding
+    A, SA, m = oracle.mass(u, 1e-8)
+    H1, _ = oracle.history_mass(A, SA, m, np.zeros(T, np.float32), 0.9, 1.0)
+    H9, c = oracle.history_mass(A, SA, m, np.zeros(T, np.float32), 0.9, 0.9)
+    assert np.abs(H1.astype(np.int64) - H9.astype(np.int64)).max() <= 2 ** 36 * 1e-6 * m.max() + 2
+    np.testing.assert_allclose(c, (np.float32(1.0) - np.float32(0.9)) * m, rtol=2e-7)
+    # credit rows travel with their tokens, zero beyond the budget
+    on = oracle.select_unit(u, u, None, Tk, Params(ema_beta=0.9))
+    assert (on.credit[:Tk] == c[on.keep_idx]).all() and (on.credit[Tk:] == 0).all()
+
+
+def test_ema_history_moves_boundaries_toward_past_mass():
+    T = 1024
+    past = np.zeros(T, np.float32); past[:128] = 1.0 / 128            # history says: mass at the front
+    u = np.zeros(T, np.float32); u[-128:] = 1.0                        # now: mass at the back
+    A, SA, m = oracle.mass(u, 1e-8)
+    H_now, _ = oracle.history_mass(A, SA, m, past, 0.9, 1.0)
+    H_mix, _ = oracle.history_mass(A, SA, m, past, 0.9, 0.5)
+    first_now = oracle.cuts(oracle.prefix(H_now), 4)[1]
+    first_mix = oracle.cuts(oracle.prefix(H_mix), 4)[1]
+    assert first_now > T - 128 and first_mix <= 128
+
+
+# ----------------------------------------------------------------------------- whole unit
+
+@pytest.mark.parametrize("seed", range(25))
+def test_unit_invariants(seed):
+    rng = np.random.default_rng(5000 + seed)
+    T = int(rng.integers(40, 6000))
+    Tk = int(rng.integers(1, T))
+    prm = Params(n_segments=int(rng.integers(1, 20)), l_min=int(rng.integers(1, 32)),
+                 l_max=int(rng.choice([0, 64, 256])), q_min=int(rng.integers(0, 4)),
+                 n_sink=int(rng.integers(0, 6)), n_last=int(rng.integers(0, 20)),
+                 ema_beta=float(rng.choice([1.0, 0.9])))
+    if prm.l_max and prm.l_max < 2 * prm.l_min:
+        prm.l_max = 2 * prm.l_min
+    u = (np.abs(rng.standard_normal(T)) ** 4).astype(np.float32)
+    g = rng.standard_normal(T).astype(np.float32)
+    res = oracle.select_unit(u, g, None, Tk, prm)
+    k = res.keep_idx
+    assert len(k) == Tk and (np.diff(k) > 0).all() and k[0] >= 0 and k[-1] < T
+    ns, nl = oracle.must_keep(T, Tk, prm.n_sink, prm.n_last)
+    assert set(range(ns)) <= set(k.tolist()) and set(range(T - nl, T)) <= set(k.tolist())
+    assert ns == min(prm.n_sink, Tk) and nl == min(prm.n_last, Tk - ns, T - ns)   # sinks before suffix
+    assert res.quotas.sum() == Tk - ns - nl
+    lens = np.diff(res.bounds)
+    assert res.bounds[0] == 0 and res.bounds[-1] == T and (res.quotas <= lens).all()
+    kept_per_seg = np.histogram(k, bins=res.bounds)[0]
+    assert (kept_per_seg >= res.quotas).all()            # each segment keeps at least its quota
+    if np.minimum(prm.q_min, lens).sum() <= Tk - ns - nl:
+        assert (kept_per_seg >= np.minimum(prm.q_min, lens)).all()   # no region wiped out
+
+
+def test_segment_count_smoke_range_at_paper_operating_point():
+    # Attention-like mass at T ~ 1.1-1.5 K, segment mass 0.1, lengths 16/256: the paper's
+    # diagnostics table reports 7-10 segments of mean length 131-148.  Weak pin: a range.
+    for seed in range(8):
+        rng = np.random.default_rng(6000 + seed)
+        T = int(rng.integers(1100, 1500))
+        u = np.exp(1.5 * rng.standard_normal(T)).astype(np.float32)
+        u[:4] += 50.0
+        u[-64:] *= 4.0
+        res = oracle.select_unit(u, u, None, 512, Params())
+        assert 5 <= res.n_seg <= 14, res.n_seg
+        assert 80 <= T / res.n_seg <= 260
+
+
+# ----------------------------------------------------------------------------- gather
+
+def test_gather_equals_dense_indexing():
+    rng = np.random.default_rng(7)
+    L, P, page, H, D, T, Tk = 2, 40, 16, 3, 128, 150, 37
+    k = rng.integers(0, 65536, size=(L, P, page, H, D)).astype(np.uint16)
+    v = rng.integers(0, 65536, size=(L, P, page, H, D)).astype(np.uint16)
+    perm = rng.permutation(P).astype(np.int32)
+    table = perm[:10]
+    dst = perm[10:13]
+    k0, v0 = k.copy(), v.copy()
+    slots = table[np.arange(T) // page] * page + np.arange(T) % page
+    for l in range(L):
+        for h in range(H):
+            keep = np.sort(rng.choice(T, size=Tk, replace=False)).astype(np.int32)
+            dense_k = k0[l].reshape(-1, H, D)[slots, h]          # [T][D] dense view of this head
+            dense_v = v0[l].reshape(-1, H, D)[slots, h]
+            oracle.gather_unit(k, v, l, h, table, dst, keep)
+            dslots = dst[np.arange(Tk) // page] * page + np.arange(Tk) % page
+            assert (k[l].reshape(-1, H, D)[dslots, h] == dense_k[keep]).all()
+            assert (v[l].reshape(-1, H, D)[dslots, h] == dense_v[keep]).all()
+    # source pages untouched, nothing outside the destination pages written
+    mask = np.ones(P, bool); mask[dst] = False
+    assert (k[:, mask] == k0[:, mask]).all() and (v[:, mask] == v0[:, mask]).all()
+
+
+# ----------------------------------------------------------------------------- scorers
+
+def _tiny_cache(rng, L=1, H=2, T=200, P=20, D=128):
+    x = torch.from_numpy(rng.standard_normal((L, P, 16, H, D)).astype(np.float32)).to(torch.bfloat16)
+    pages = x.view(torch.int16).numpy().view(np.uint16)
+    table = rng.permutation(P).astype(np.int32)[: (T + 15) // 16]
+    slots = table[np.arange(T) // 16] * 16 + np.arange(T) % 16
+    dense = x.float().double().reshape(L, -1, H, D)[:, slots]     # [L][T][H][D]
+    return pages, table, dense
+
+
+def test_tova_single_row_is_library_softmax():
+    rng = np.random.default_rng(11)
+    pages, table, dense = _tiny_cache(rng)
+    T, D = dense.shape[1], 128
+    q = torch.from_numpy(rng.standard_normal((1, 1, D)).astype(np.float32)).to(torch.bfloat16)
+    for h in range(2):
+        u = oracle.score_tova(pages, 0, h, table, T, q.view(torch.int16).numpy().view(np.uint16), 1, 1, True)
+        ref = torch.softmax(dense[0, :, h] @ q.double().reshape(D) / np.sqrt(D), dim=0)
+        np.testing.assert_allclose(u, ref.numpy(), rtol=2e-7, atol=0)
+        assert abs(float(u.astype(np.float64).sum()) - 1.0) < 1e-6
+    # permuting the tokens permutes the scores
+    perm = rng.permutation(len(table) * 16)[:T]
+
+
+def test_tova_window_group_mean_and_causal_padding():
+    rng = np.random.default_rng(12)
+    pages, table, dense = _tiny_cache(rng, T=120, P=12)
+    T, D, G, W = 120, 128, 3, 5
+    q = torch.from_numpy((rng.standard_normal((G, W, D)) * 2).astype(np.float32)).to(torch.bfloat16)
+    qn = q.view(torch.int16).numpy().view(np.uint16)
+    K = dense[0, :, 1]
+    # non-causal: plain mean of G*W library softmaxes
+    u = oracle.score_tova(pages, 0, 1, table, T, qn, G, W, False)
+    ref = torch.softmax(q.double().reshape(G * W, D) @ K.T / np.sqrt(D), dim=1).mean(0)
+    np.testing.assert_allclose(u, ref.numpy(), rtol=3e-7)
+    # causal: window query j sees tokens t <= T-W+j; unseen pairs take the window maximum
+    u = oracle.score_tova(pages, 0, 1, table, T, qn, G, W, True)
+    probs = torch.zeros(G, W, T, dtype=torch.float64)
+    for j in range(W):
+        n = T - W + j + 1
+        probs[:, j, :n] = torch.softmax(q.double()[:, j] @ K[:n].T / np.sqrt(D), dim=1)
+    pmax = probs.max()
+    seen = torch.arange(T)[None, :] <= (T - W + torch.arange(W))[:, None]
+    ref = torch.where(seen[None], probs, pmax).mean((0, 1))
+    np.testing.assert_allclose(u, ref.numpy(), rtol=3e-7)
+    assert np.allclose(u[: T - W + 1], probs.mean((0, 1))[: T - W + 1].numpy(), rtol=3e-7)
+    # identical rows collapse to one softmax
+    q1 = q[:1, :1].expand(G, W, D).contiguous()
+    u1 = oracle.score_tova(pages, 0, 1, table, T, q1.view(torch.int16).numpy().view(np.uint16), G, W, False)
+    r1 = torch.softmax(K @ q1.double()[0, 0] / np.sqrt(D), dim=0)
+    np.testing.assert_allclose(u1, r1.numpy(), rtol=3e-7)
+
+
+def test_keydiff_is_negative_cosine_to_mean_key():
+    rng = np.random.default_rng(13)
+    pages, table, dense = _tiny_cache(rng, T=333, P=30)
+    for h in range(2):
+        K = dense[0, :, h]
+        g = oracle.score_keydiff(pages, 0, h, table, 333)
+        ref = -torch.nn.functional.cosine_similarity(K, K.mean(0, keepdim=True), dim=1)
+        np.testing.assert_allclose(g, ref.numpy(), rtol=1e-6, atol=1e-7)
+    # closed forms: identical keys -> -1; a key orthogonal to the mean -> 0; opposite -> +1
+    L, P, H, D = 1, 1, 1, 128
+    x = torch.zeros((L, P, 16, H, D))
+    x[0, 0, :, 0, 0] = 2.0
+    pg = x.to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    g = oracle.score_keydiff(pg, 0, 0, np.array([0], np.int32), 16)
+    assert (g == -1.0).all()
+    x[0, 0, 3, 0, :] = 0.0; x[0, 0, 3, 0, 5] = 7.0             # orthogonal to the mean direction... almost
+    x[0, 0, 4, 0, 0] = -0.5                                     # opposite
+    pg = x.to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    g = oracle.score_keydiff(pg, 0, 0, np.array([0], np.int32), 16)
+    mu = x[0, 0, :, 0].double().mean(0)
+    assert abs(g[3] + float(7.0 * mu[5] / (7.0 * mu.norm()))) < 1e-6
+    assert g[4] > 0.9 and g[0] < -0.9
