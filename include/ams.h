@@ -1,0 +1,152 @@
+/*
+ * libams — the periodic Adaptive Mass-Segmented (AMS) KV-compression step on a
+ * paged bf16 KV cache, for NVIDIA B200 (sm_100a).  C ABI: plain pointers and
+ * sizes only.  Every pointer marked DEVICE is device memory owned by the caller;
+ * the library allocates and frees no device memory.  `stream` arguments are
+ * `cudaStream_t` values passed as `void*`.
+ *
+ * One call of ams_compress performs, for every layer, sequence and KV head,
+ * Algorithm 1 of the paper followed by the paged head-wise compaction of its
+ * serving appendix:
+ *   1. score every cached token (TOVA-style observation-window softmax averaged
+ *      over the GQA group — Section 3.2 and Algorithm 1 step 1 — or a key-only
+ *      KeyDiff-style score);
+ *   2. turn usage into the normalised quality mass (Eq. 1), mix it with the EMA
+ *      credit carried across events (Section 3.3, "EMA credit"; Algorithm 1 step 2);
+ *   3. prefix-sum the mass, cut at multiples of the segment mass, merge short and
+ *      split long segments (Section 3.3, "Mass-based adaptive segmentation";
+ *      Algorithm 1 step 3);
+ *   4. give each segment its quota of the budget (Section 3.3, "Segment-wise quota
+ *      allocation"; Algorithm 1 step 4);
+ *   5. keep the top-q_i tokens of each segment, the must-keep prefix/suffix, and
+ *      backfill to exactly `budget` positions (Algorithm 1 step 5);
+ *   6. move the kept K/V rows of every head into replacement pages and rewrite the
+ *      block-table row and the sequence length (the two display equations and the
+ *      runtime routine of the paged-KV appendix).
+ *
+ * Layouts (all contiguous, row-major):
+ *   k_pages, v_pages : bf16  [n_layers][num_pages][16][n_kv_heads][128]
+ *   block_table      : int32 [batch][block_table_stride]  page ids shared by all layers and heads
+ *   seq_lens         : int32 [batch]
+ *   obs_queries      : bf16  [n_layers][batch][n_q_heads][window][128]; window query j is the
+ *                      decode query at position seq_len - window + j
+ *   ema_state        : fp32  [n_layers][max_batch][n_kv_heads][max_seq_len]  credit per cached row
+ *   dst_pages        : int32 [batch][ceil(budget/16)]  free pages that receive the kept rows
+ *   per-unit views   : [n_layers][batch][n_kv_heads][...]
+ *
+ * Decisions (cut positions, quotas, kept indices) are taken in integer arithmetic
+ * on fixed-point images of the mass, so they do not depend on summation order.
+ *
+ * Errors: every function returns AMS_OK (0) or a negative code.  Calls are
+ * asynchronous on `stream`; conditions found on the device (a sequence longer
+ * than max_seq_len, a window longer than a sequence, a bounded wait that ran out)
+ * skip the affected work and are reported by ams_get_status.
+ */
+#ifndef AMS_H_
+#define AMS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    AMS_OK = 0,
+    AMS_ERR_INVALID_ARG = -1, /* null pointer, size out of range, budget < 1, ...            */
+    AMS_ERR_UNSUPPORTED = -2, /* head_dim != 128, page_size != 16, n_q_heads % n_kv_heads    */
+    AMS_ERR_CAPACITY = -3,    /* workspace too small, or a device-side capacity was exceeded  */
+    AMS_ERR_CUDA = -4,        /* a CUDA runtime call or launch failed                         */
+    AMS_ERR_TIMEOUT = -5,     /* a bounded device-side wait expired                           */
+    AMS_ERR_INTERNAL = -6     /* a device-side consistency check failed                       */
+};
+
+enum { AMS_SCORER_TOVA = 0, AMS_SCORER_KEYDIFF = 1, AMS_SCORER_EXTERNAL = 2 };
+
+typedef struct ams_state ams_state; /* opaque host handle */
+
+typedef struct {
+    int32_t n_layers, n_q_heads, n_kv_heads; /* GQA group = n_q_heads / n_kv_heads           */
+    int32_t head_dim;                        /* must be 128                                   */
+    int32_t page_size;                       /* must be 16                                    */
+    int32_t max_batch;                       /* capacity: sequences per call                  */
+    int32_t max_seq_len;                     /* capacity: tokens per sequence, <= 131072      */
+    int32_t max_window;                      /* capacity: observation queries                 */
+    int32_t max_budget;                      /* capacity: tokens kept per head                */
+    int32_t max_segments;                    /* capacity: n_segments                          */
+    int32_t l_min, l_max;                    /* segment length bounds; l_max = 0: no split    */
+    int32_t q_min;                           /* guaranteed quota per segment                  */
+    int32_t n_sink, n_last;                  /* must-keep prefix / suffix                     */
+    float ema_lambda;                        /* credit decay, in [0, 1)                       */
+    float ema_beta;                          /* weight of the current mass; 1 = credit unused */
+    float eps;                               /* Eq. 1 epsilon, > 0                            */
+    int32_t causal_window;                   /* 1: window query j sees tokens <= T - W + j    */
+} ams_config;
+
+/* Optional device outputs for inspection and tests; any member may be NULL.
+ * T = max_seq_len, C = ams_segment_capacity(cfg).  Units that were skipped
+ * (seq_len <= budget) are left untouched. */
+typedef struct {
+    float *scores;       /* [L][batch][H][T]   base scores g (= usage u)                    */
+    float *mass;         /* [L][batch][H][T]   Eq. 1 mass of the current event              */
+    int32_t *n_segments; /* [L][batch][H]      segments after merge and split               */
+    int32_t *seg_bounds; /* [L][batch][H][C+1] boundaries a_0 = 0 < ... < a_n = seq_len     */
+    int32_t *quotas;     /* [L][batch][H][C]                                                 */
+    int32_t *keep_idx;   /* [L][batch][H][budget] kept positions, ascending                 */
+} ams_debug_views;
+
+/* Paper defaults: segment mass 0.1 (n_segments = 10 is passed per call), lengths
+ * 16 / 256, q_min 1, lambda = beta = 0.9, 4 sinks; n_last 16, eps 1e-8.  Geometry
+ * and capacities are zeroed and must be filled by the caller. */
+void ams_config_default(ams_config *cfg);
+
+/* Sizes of the caller-allocated device buffers; 0 if the configuration is invalid. */
+size_t ams_ema_state_bytes(const ams_config *cfg);
+size_t ams_workspace_bytes(const ams_config *cfg);
+/* Per-unit capacity C of the segment views: max_segments + 2*floor(max_seq_len/l_max) + 4. */
+int32_t ams_segment_capacity(const ams_config *cfg);
+
+/* Creates the host handle, zero-fills ema_state (DEVICE, ams_ema_state_bytes) on
+ * `stream`, and adopts `workspace` (DEVICE, >= ams_workspace_bytes, 256-byte
+ * aligned) as scratch for later calls.  Both buffers must outlive the handle. */
+int ams_init_state(const ams_config *cfg, void *ema_state, void *workspace, size_t workspace_bytes,
+                   void *stream, ams_state **out);
+
+/* One compression event (see the file header).  All pointers DEVICE.
+ *  k_pages, v_pages : read at the pages named by block_table, written at the pages named by
+ *                     dst_pages (which must not overlap the live pages); nothing else is touched.
+ *  num_pages        : pages per layer of the pool.
+ *  block_table, seq_lens : updated in place for every sequence with seq_len > budget:
+ *                     row <- dst_pages row followed by -1, length <- budget.  Sequences with
+ *                     seq_len <= budget are left as they are (nothing to evict).
+ *  obs_queries, window : may be NULL / 0 for AMS_SCORER_KEYDIFF and AMS_SCORER_EXTERNAL.
+ *  ema_state        : the buffer given to ams_init_state (or a restored copy of it).
+ *  n_segments       : S, the number of mass quantiles (segment mass 1/S), 1..max_segments.
+ *  ext_scores       : AMS_SCORER_EXTERNAL only: fp32 [L][batch][H][max_seq_len] scores used both
+ *                     as usage and as base scores.
+ *  dbg              : optional views, or NULL.
+ * Calls on the same handle share the workspace and must not overlap on the GPU. */
+int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages, int32_t *block_table,
+                 int32_t block_table_stride, int32_t *seq_lens, int32_t batch, const void *obs_queries,
+                 int32_t window, void *ema_state, int32_t budget, int32_t n_segments, int32_t scorer_id,
+                 const int32_t *dst_pages, const float *ext_scores, const ams_debug_views *dbg,
+                 void *stream);
+
+/* Synchronises `stream`, then returns and clears the device status: AMS_OK or the
+ * first device-side error.  detail[0..3] (host, may be NULL) receive the code, the
+ * unit index and two values describing it. */
+int ams_get_status(ams_state *st, void *stream, int32_t *detail);
+
+/* Number of kernels the last ams_compress on this handle launched. */
+int32_t ams_last_launch_count(const ams_state *st);
+
+/* Releases the host handle only. */
+int ams_free(ams_state *st);
+
+const char *ams_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AMS_H_ */

@@ -1,0 +1,204 @@
+"""ctypes binding of libams.so: argument marshalling only.
+
+Every step of the compression path runs inside the library's CUDA kernels; this
+module turns torch tensors into device pointers and owns the two buffers the
+library asks the caller to allocate (EMA credit state and workspace).  If the
+library is missing or fails to load, importing the functions raises: there is no
+CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libams.so")
+
+AMS_OK = 0
+AMS_ERR_INVALID_ARG, AMS_ERR_UNSUPPORTED, AMS_ERR_CAPACITY = -1, -2, -3
+AMS_ERR_CUDA, AMS_ERR_TIMEOUT, AMS_ERR_INTERNAL = -4, -5, -6
+AMS_SCORER_TOVA, AMS_SCORER_KEYDIFF, AMS_SCORER_EXTERNAL = 0, 1, 2
+
+EXPORTS = ["ams_config_default", "ams_ema_state_bytes", "ams_workspace_bytes", "ams_segment_capacity",
+           "ams_init_state", "ams_compress", "ams_get_status", "ams_last_launch_count", "ams_free",
+           "ams_strerror"]
+
+
+class AmsConfig(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("n_layers", "n_q_heads", "n_kv_heads", "head_dim", "page_size", "max_batch", "max_seq_len",
+                 "max_window", "max_budget", "max_segments", "l_min", "l_max", "q_min", "n_sink", "n_last")] + \
+               [("ema_lambda", ctypes.c_float), ("ema_beta", ctypes.c_float), ("eps", ctypes.c_float),
+                ("causal_window", ctypes.c_int32)]
+
+
+class AmsDebugViews(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("scores", "mass", "n_segments", "seg_bounds", "quotas", "keep_idx")]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libams.so (must have been built: `python -m paper_2605_23200_b200.build`)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} not built; run paper_2605_23200_b200/build.py (no CPU fallback exists)")
+        L = ctypes.CDLL(LIB_PATH)
+        L.ams_config_default.argtypes = [ctypes.POINTER(AmsConfig)]
+        L.ams_config_default.restype = None
+        for f in ("ams_ema_state_bytes", "ams_workspace_bytes"):
+            getattr(L, f).argtypes = [ctypes.POINTER(AmsConfig)]
+            getattr(L, f).restype = ctypes.c_size_t
+        L.ams_segment_capacity.argtypes = [ctypes.POINTER(AmsConfig)]
+        L.ams_segment_capacity.restype = ctypes.c_int32
+        L.ams_init_state.argtypes = [ctypes.POINTER(AmsConfig), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t,
+                                     ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p)]
+        L.ams_init_state.restype = ctypes.c_int
+        L.ams_compress.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
+                                   ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_int32,
+                                   ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_int32,
+                                   ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
+                                   ctypes.POINTER(AmsDebugViews), ctypes.c_void_p]
+        L.ams_compress.restype = ctypes.c_int
+        L.ams_get_status.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32)]
+        L.ams_get_status.restype = ctypes.c_int
+        L.ams_last_launch_count.argtypes = [ctypes.c_void_p]
+        L.ams_last_launch_count.restype = ctypes.c_int32
+        L.ams_free.argtypes = [ctypes.c_void_p]
+        L.ams_free.restype = ctypes.c_int
+        L.ams_strerror.argtypes = [ctypes.c_int]
+        L.ams_strerror.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().ams_strerror(code).decode()
+
+
+class AmsError(RuntimeError):
+    def __init__(self, code: int, where: str, detail=None):
+        self.code = code
+        self.detail = detail
+        super().__init__(f"{where}: {strerror(code)} ({code})" + (f" detail={detail}" if detail else ""))
+
+
+def default_config(**kw) -> AmsConfig:
+    cfg = AmsConfig()
+    lib().ams_config_default(ctypes.byref(cfg))
+    for k, v in kw.items():
+        if not hasattr(cfg, k):
+            raise AttributeError(k)
+        setattr(cfg, k, v)
+    return cfg
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+@dataclass
+class DebugViews:
+    """Device tensors that receive the library's intermediate results."""
+    scores: torch.Tensor
+    mass: torch.Tensor
+    n_segments: torch.Tensor
+    seg_bounds: torch.Tensor
+    quotas: torch.Tensor
+    keep_idx: torch.Tensor
+
+    def c(self) -> AmsDebugViews:
+        return AmsDebugViews(*(t.data_ptr() for t in
+                               (self.scores, self.mass, self.n_segments, self.seg_bounds, self.quotas, self.keep_idx)))
+
+
+class AmsCompressor:
+    """Owns an `ams_state` handle together with the EMA credit and workspace tensors."""
+
+    def __init__(self, cfg: AmsConfig, device="cuda:0", stream: torch.cuda.Stream | None = None):
+        L = lib()
+        self.cfg = cfg
+        self.device = torch.device(device)
+        ema_bytes = L.ams_ema_state_bytes(ctypes.byref(cfg))
+        ws_bytes = L.ams_workspace_bytes(ctypes.byref(cfg))
+        if ema_bytes == 0 or ws_bytes == 0:
+            raise AmsError(AMS_ERR_INVALID_ARG, "ams_config")
+        self.seg_cap = L.ams_segment_capacity(ctypes.byref(cfg))
+        self.ema_state = torch.empty((cfg.n_layers, cfg.max_batch, cfg.n_kv_heads, cfg.max_seq_len),
+                                     dtype=torch.float32, device=self.device)
+        self.workspace = torch.empty(ws_bytes + 256, dtype=torch.uint8, device=self.device)
+        off = (-self.workspace.data_ptr()) % 256
+        self._ws_ptr = self.workspace.data_ptr() + off
+        self._ws_bytes = ws_bytes
+        handle = ctypes.c_void_p()
+        s = stream or torch.cuda.current_stream(self.device)
+        rc = L.ams_init_state(ctypes.byref(cfg), _ptr(self.ema_state), ctypes.c_void_p(self._ws_ptr), ws_bytes,
+                              ctypes.c_void_p(s.cuda_stream), ctypes.byref(handle))
+        if rc != AMS_OK:
+            raise AmsError(rc, "ams_init_state")
+        self._h = handle
+
+    def make_debug_views(self, batch: int, budget: int) -> DebugViews:
+        c, dev = self.cfg, self.device
+        U = (c.n_layers, batch, c.n_kv_heads)
+        return DebugViews(torch.zeros(U + (c.max_seq_len,), dtype=torch.float32, device=dev),
+                          torch.zeros(U + (c.max_seq_len,), dtype=torch.float32, device=dev),
+                          torch.zeros(U, dtype=torch.int32, device=dev),
+                          torch.zeros(U + (self.seg_cap + 1,), dtype=torch.int32, device=dev),
+                          torch.zeros(U + (self.seg_cap,), dtype=torch.int32, device=dev),
+                          torch.zeros(U + (budget,), dtype=torch.int32, device=dev))
+
+    def compress(self, k_pages, v_pages, block_table, seq_lens, obs_queries, budget, n_segments, scorer_id,
+                 dst_pages, *, ext_scores=None, dbg: DebugViews | None = None, ema_state=None,
+                 stream: torch.cuda.Stream | None = None) -> None:
+        """Enqueues one compression event on `stream` (default: torch's current stream)."""
+        assert k_pages.is_contiguous() and v_pages.is_contiguous() and block_table.is_contiguous()
+        assert k_pages.dtype == torch.bfloat16 and block_table.dtype == torch.int32 and seq_lens.dtype == torch.int32
+        assert dst_pages.dtype == torch.int32 and dst_pages.is_contiguous()
+        s = stream or torch.cuda.current_stream(self.device)
+        window = 0 if obs_queries is None else obs_queries.shape[3]
+        ema = self.ema_state if ema_state is None else ema_state
+        views = dbg.c() if dbg is not None else None
+        rc = lib().ams_compress(self._h, _ptr(k_pages), _ptr(v_pages), k_pages.shape[1], _ptr(block_table),
+                                block_table.shape[1], _ptr(seq_lens), seq_lens.shape[0], _ptr(obs_queries), window,
+                                _ptr(ema), budget, n_segments, scorer_id, _ptr(dst_pages), _ptr(ext_scores),
+                                ctypes.byref(views) if views is not None else None, ctypes.c_void_p(s.cuda_stream))
+        if rc != AMS_OK:
+            raise AmsError(rc, "ams_compress")
+
+    def status(self, stream: torch.cuda.Stream | None = None, check: bool = True):
+        s = stream or torch.cuda.current_stream(self.device)
+        detail = (ctypes.c_int32 * 4)()
+        rc = lib().ams_get_status(self._h, ctypes.c_void_p(s.cuda_stream), detail)
+        if check and rc != AMS_OK:
+            raise AmsError(rc, "device status", list(detail))
+        return rc, list(detail)
+
+    @property
+    def last_launch_count(self) -> int:
+        return lib().ams_last_launch_count(self._h)
+
+    def close(self) -> None:
+        if getattr(self, "_h", None):
+            lib().ams_free(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def config_for(wl, **kw) -> AmsConfig:
+    """Library configuration matching an `inputs.Workload`."""
+    return default_config(n_layers=wl.layers_resident, n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads,
+                          max_batch=wl.batch, max_seq_len=wl.max_seq_len, max_window=max(wl.window, 0),
+                          max_budget=wl.budget, max_segments=max(wl.n_segments, 1), l_min=wl.l_min, l_max=wl.l_max,
+                          q_min=wl.q_min, n_sink=wl.n_sink, n_last=wl.n_last, ema_lambda=wl.ema_lambda,
+                          ema_beta=wl.ema_beta, eps=wl.eps, **kw)

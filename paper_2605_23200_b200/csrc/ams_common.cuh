@@ -1,0 +1,175 @@
+// Shared device-side definitions of libams (sm_100a).  Nothing here is used by, or
+// shared with, the CPU oracle.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/ams.h"
+
+namespace ams {
+
+constexpr int kHeadDim = 128;
+constexpr int kPage = 16;
+constexpr int kFixBits = 36;          // fractional bits of the fixed-point mass images
+constexpr int kRowBytes = kHeadDim * 2;
+
+typedef unsigned long long u64;
+
+// Everything a kernel of one ams_compress call needs; passed by value.
+struct DevParams {
+    // geometry of the call
+    int L, B, Bmax, H, G, W, rows;    // rows = G * W query rows per KV head
+    int T_cap, seg_cap, Tk, S, n_dst; // n_dst = ceil(Tk / 16)
+    int l_min, l_max, q_min, n_sink, n_last, causal;
+    float lambda, beta, eps;
+    // caller buffers
+    __nv_bfloat16 *k_pages, *v_pages;
+    long long num_pages;
+    int *block_table;
+    int bt_stride;
+    int *seq_lens;
+    const __nv_bfloat16 *q;           // [L][B][H*G][W][128]
+    float *ema;                       // [L][Bmax][H][T_cap]
+    const int *dst_pages;             // [B][n_dst]
+    // per-unit working arrays, [L*B*H][...]
+    const float *usage;               // u: what the mass is built from
+    float *scores;                    // g: what segments rank by (== usage unless external)
+    u64 *cbuf;                        // [T_cap]  integer mass, then its inclusive prefix sum
+    unsigned char *flags;             // [T_cap]  1 = kept
+    int *n_seg;                       // [1]
+    int *seg_bounds;                  // [seg_cap + 1]
+    int *quotas;                      // [seg_cap]
+    int *keep_idx;                    // [Tk]
+    float *mass_dbg;                  // [T_cap] or null
+    // scorer scratch
+    float *part;                      // per (unit, slice) partials
+    float *fin;                       // per unit finals
+    int slice_len, n_slices, rows_pad;
+    int *status;                      // [4]: code, unit, a, b
+};
+
+__device__ __forceinline__ void set_status(int *status, int code, int unit, int a, int b)
+{
+    if (atomicCAS(status, 0, code) == 0) {
+        status[1] = unit;
+        status[2] = a;
+        status[3] = b;
+    }
+}
+
+// Element offset of the 128-wide row (layer, page, slot, head) in a page pool.
+__device__ __forceinline__ size_t row_offset(const DevParams &p, int layer, int page, int slot, int h)
+{
+    return ((((size_t)layer * (size_t)p.num_pages + (size_t)page) * kPage + slot) * p.H + h) * kHeadDim;
+}
+
+// ------------------------------------------------------------------ block primitives
+// All take a shared scratch array of at least 33 u64 and work for any block size
+// that is a multiple of 32 (<= 1024).  Each ends with the result in every thread.
+
+__device__ __forceinline__ u64 warp_sum_u64(u64 v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ u64 block_sum_u64(u64 v, u64 *scratch)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    v = warp_sum_u64(v);
+    __syncthreads();
+    if (lane == 0) scratch[warp] = v;
+    __syncthreads();
+    if (warp == 0) {
+        u64 x = lane < nw ? scratch[lane] : 0ull;
+        x = warp_sum_u64(x);
+        if (lane == 0) scratch[32] = x;
+    }
+    __syncthreads();
+    return scratch[32];
+}
+
+__device__ __forceinline__ long long block_sum_i64(long long v, u64 *scratch)
+{
+    return (long long)block_sum_u64((u64)v, scratch);
+}
+
+__device__ __forceinline__ float block_max_f32(float v, u64 *scratch)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    __syncthreads();
+    if (lane == 0) scratch[warp] = (u64)__float_as_uint(v);
+    __syncthreads();
+    if (warp == 0) {
+        float x = lane < nw ? __uint_as_float((unsigned)scratch[lane]) : 0.0f;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
+        if (lane == 0) scratch[32] = (u64)__float_as_uint(x);
+    }
+    __syncthreads();
+    return __uint_as_float((unsigned)scratch[32]);
+}
+
+// Exclusive prefix of v over the threads of the block; *total receives the block sum.
+__device__ __forceinline__ u64 block_excl_scan_u64(u64 v, u64 *scratch, u64 *total)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    u64 inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        u64 y = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += y;
+    }
+    __syncthreads();
+    if (lane == 31) scratch[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        u64 x = lane < nw ? scratch[lane] : 0ull;
+        u64 xi = x;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            u64 y = __shfl_up_sync(0xffffffffu, xi, o);
+            if (lane >= o) xi += y;
+        }
+        scratch[lane] = xi - x; // exclusive prefix of the warp sums
+        if (lane == 31) scratch[32] = xi;
+    }
+    __syncthreads();
+    *total = scratch[32];
+    return scratch[warp] + inc - v;
+}
+
+// Order-preserving image of an fp32 score; NaN ranks below everything.
+__device__ __forceinline__ unsigned score_key(float x)
+{
+    const unsigned b = __float_as_uint(x);
+    if ((b & 0x7fffffffu) > 0x7f800000u) return 0u;
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+// bf16 pair -> two fp32 (exact).
+__device__ __forceinline__ float bf16_lo(unsigned w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(unsigned w) { return __uint_as_float(w & 0xffff0000u); }
+
+// 16-byte global load that does not pollute L1 (streamed once per phase).
+__device__ __forceinline__ uint4 ld_stream16(const void *ptr)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(ptr));
+    return v;
+}
+
+// Host-side launchers (one per translation unit).
+int tova_rows_block(int rows); // query rows handled per pass of the TOVA kernel (8..128)
+int launch_score_tova(const DevParams &p, cudaStream_t s, int *launches);
+int launch_score_keydiff(const DevParams &p, cudaStream_t s, int *launches);
+int launch_segment_select(const DevParams &p, cudaStream_t s, int *launches);
+int launch_gather(const DevParams &p, cudaStream_t s, int *launches);
+
+} // namespace ams

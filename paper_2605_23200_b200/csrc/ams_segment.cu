@@ -1,0 +1,493 @@
+// Mass, EMA credit, prefix scan, cuts, merge/split, quotas, segmented radix select,
+// must-keep, backfill and ordered index compaction: Algorithm 1 steps 1-5 of the
+// paper for one (layer, sequence, KV head) per thread block.
+//
+// Every decision is integer arithmetic on fixed-point images of the mass (kFixBits
+// fractional bits) and every floating-point step is a single round-to-nearest
+// operation, so the result does not depend on how the block orders its sums.
+#include <float.h>
+
+#include "ams_common.cuh"
+
+namespace ams {
+
+namespace {
+
+__device__ __forceinline__ float weight_of(float u, float eps)
+{
+    // Eq. 1 numerator: max(u, 0) + eps; NaN counts as 0, +inf as FLT_MAX.
+    float v = __fadd_rn(fmaxf(u, 0.0f), eps);
+    if (!(v <= FLT_MAX)) v = FLT_MAX;
+    return v;
+}
+
+// 2^(kFixBits - (ilogb(mx) + 1)) as a double; mx > 0 (any fp32, subnormals included).
+__device__ __forceinline__ double fix_scale(float mx)
+{
+    const long long bits = __double_as_longlong((double)mx);
+    const int e = (int)((bits >> 52) & 0x7ff) - 1023 + 1;
+    return __longlong_as_double((long long)(1023 + kFixBits - e) << 52);
+}
+
+__device__ __forceinline__ u64 to_fixed(float x, double scale)
+{
+    return (u64)__double2ull_rd(__dmul_rn((double)x, scale));
+}
+
+// min(floor(C * S / SH), S - 1): index of the last mass quantile reached at prefix C.
+__device__ __forceinline__ int quantile_of(u64 C, u64 S, u64 SH)
+{
+    const u64 k = (C * S) / SH;
+    return (int)(k < S - 1 ? k : S - 1);
+}
+
+struct Smem {
+    u64 scratch[40];
+    int bcast[8];
+};
+
+// Gives `D` (> 0) tokens to segments one per visit, cycling in the visiting order,
+// where segment i can take at most cap[i].  Closed form of the cycle: every segment
+// receives min(cap, k) with k the largest level whose total fits, and the first
+// `rem` segments (in visiting order) that still have room receive one more.
+// heavy_first: order (M desc, i asc); otherwise (M asc, i desc).  Returns what is left.
+template <bool kHeavyFirst>
+__device__ long long distribute(long long D, const int *cap, int *give, const u64 *M, int n_seg, Smem &sm)
+{
+    const int tid = threadIdx.x, nt = blockDim.x;
+    long long cnt1 = 0, tot = 0;
+    int mx = 0;
+    for (int i = tid; i < n_seg; i += nt) {
+        cnt1 += cap[i] >= 1;
+        tot += cap[i];
+        mx = max(mx, cap[i]);
+    }
+    cnt1 = block_sum_i64(cnt1, sm.scratch);
+    tot = block_sum_i64(tot, sm.scratch);
+    mx = (int)block_max_f32((float)mx, sm.scratch); // exact below 2^24; caps are <= 2^17
+    long long level = 0, used = 0;
+    if (tot <= D) {
+        level = mx;
+        used = tot;
+    } else if (cnt1 <= D) {
+        long long lo = 1, hi = mx; // F(lo) <= D < F(hi)
+        used = cnt1;
+        while (hi - lo > 1) {
+            const long long mid = (lo + hi) >> 1;
+            long long f = 0;
+            for (int i = tid; i < n_seg; i += nt) f += min((long long)cap[i], mid);
+            f = block_sum_i64(f, sm.scratch);
+            if (f <= D) { lo = mid; used = f; } else hi = mid;
+        }
+        level = lo;
+    }
+    const long long rem = D - used;
+    for (int i = tid; i < n_seg; i += nt) {
+        int g = (int)min((long long)cap[i], level);
+        if (rem > 0 && cap[i] > level) {
+            long long rank = 0;
+            const u64 Mi = M[i];
+            for (int j = 0; j < n_seg; ++j) {
+                if (cap[j] <= level) continue;
+                const u64 Mj = M[j];
+                const bool before = kHeavyFirst ? (Mj > Mi || (Mj == Mi && j < i)) : (Mj < Mi || (Mj == Mi && j > i));
+                rank += before;
+            }
+            if (rank < rem) ++g;
+        }
+        give[i] = g;
+    }
+    __syncthreads();
+    return tot <= D ? D - tot : 0;
+}
+
+// k-th largest (k >= 1) of the keys selected by `pred` among positions [a, b), found by
+// a 4-pass, 8-bit radix select with a shared histogram.  The calling group is a warp
+// (kBlock = false) or the whole block (kBlock = true).  On return *thr is that key,
+// *take the number of positions equal to it that belong to the top k, and *ties the
+// number of positions equal to it.
+template <bool kBlock, typename Pred>
+__device__ void radix_select(const float *g, int a, int b, int k, int *hist, int *bc, Pred pred,
+                             unsigned *thr, int *take, int *ties)
+{
+    const int lane = threadIdx.x & 31;
+    const int gid = kBlock ? threadIdx.x : lane;
+    const int gsz = kBlock ? blockDim.x : 32;
+    unsigned prefix = 0, mask = 0;
+    int n_ties = 0;
+    for (int pass = 0; pass < 4; ++pass) {
+        const int shift = 24 - 8 * pass;
+        for (int i = gid; i < 256; i += gsz) hist[i] = 0;
+        if (kBlock) __syncthreads(); else __syncwarp();
+        for (int t = a + gid; t < b; t += gsz) {
+            if (!pred(t)) continue;
+            const unsigned key = score_key(g[t]);
+            if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
+        }
+        if (kBlock) __syncthreads(); else __syncwarp();
+        if (!kBlock || threadIdx.x < 32) {
+            // lane 0 owns the top eight bins; walk down until k positions are covered
+            int c[8], lsum = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { c[i] = hist[255 - 8 * lane - i]; lsum += c[i]; }
+            int inc = lsum;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int y = __shfl_up_sync(0xffffffffu, inc, o);
+                if (lane >= o) inc += y;
+            }
+            const int exc = inc - lsum;
+            const bool owner = exc < k && k <= inc;
+            const unsigned who = __ballot_sync(0xffffffffu, owner);
+            int digit = 0, knew = k, cnt = 0;
+            if (owner) {
+                int run = exc;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    if (run < k && k <= run + c[i]) { digit = 255 - 8 * lane - i; knew = k - run; cnt = c[i]; }
+                    run += c[i];
+                }
+            }
+            const int src = who ? __ffs(who) - 1 : 0;
+            digit = __shfl_sync(0xffffffffu, digit, src);
+            knew = __shfl_sync(0xffffffffu, knew, src);
+            cnt = __shfl_sync(0xffffffffu, cnt, src);
+            if (kBlock) { if (lane == 0) { bc[0] = digit; bc[1] = knew; bc[2] = cnt; } }
+            else { bc[0] = digit; bc[1] = knew; bc[2] = cnt; }
+            if (!kBlock) { k = knew; prefix |= (unsigned)digit << shift; n_ties = cnt; }
+        }
+        if (kBlock) {
+            __syncthreads();
+            k = bc[1];
+            prefix |= (unsigned)bc[0] << shift;
+            n_ties = bc[2];
+            __syncthreads();
+        }
+        mask |= 0xffu << shift;
+    }
+    *thr = prefix;
+    *take = k;
+    *ties = n_ties;
+}
+
+} // namespace
+
+__global__ void __launch_bounds__(1024) k_segment_select(DevParams p)
+{
+    extern __shared__ __align__(16) unsigned char dyn[];
+    __shared__ Smem sm;
+    const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
+    const int uid = blockIdx.x;
+    const int h = uid % p.H, b = (uid / p.H) % p.B, l = uid / (p.H * p.B);
+    const int T = p.seq_lens[b];
+    if (T <= p.Tk) return; // nothing to evict
+    if (T > p.T_cap) { if (tid == 0) set_status(p.status, AMS_ERR_CAPACITY, uid, T, p.T_cap); return; }
+
+    // dynamic shared memory: bounds[seg_cap+1] | quota[seg_cap] | cap[seg_cap] | give[seg_cap] | M[seg_cap]
+    //                        | raw[S+1] | merged[S+1] | pieces_off[S+1] | hist[nw*256]
+    const int sc = p.seg_cap;
+    u64 *Ms = reinterpret_cast<u64 *>(dyn);
+    int *bounds = reinterpret_cast<int *>(Ms + sc);
+    int *quota = bounds + sc + 1;
+    int *cap = quota + sc;
+    int *give = cap + sc;
+    int *raw = give + sc;
+    int *merged = raw + p.S + 1;
+    int *poff = merged + p.S + 1;
+    int *hist = poff + p.S + 1;
+
+    const float *u = p.usage + (size_t)uid * p.T_cap;
+    const float *g = p.scores + (size_t)uid * p.T_cap;
+    float *credit = p.ema + (((size_t)l * p.Bmax + b) * p.H + h) * (size_t)p.T_cap;
+    u64 *Cb = p.cbuf + (size_t)uid * p.T_cap;
+    unsigned char *flags = p.flags + (size_t)uid * p.T_cap;
+    int *keep = p.keep_idx + (size_t)uid * p.Tk;
+    float *mass_dbg = p.mass_dbg ? p.mass_dbg + (size_t)uid * p.T_cap : nullptr;
+    const bool ema_on = p.beta != 1.0f;
+    const double two_f = (double)(1ull << kFixBits);
+
+    // ---- Eq. 1 on fixed-point weights
+    float wmax = 0.0f;
+    for (int t = tid; t < T; t += nt) wmax = fmaxf(wmax, weight_of(u[t], p.eps));
+    wmax = block_max_f32(wmax, sm.scratch);
+    const double sw = fix_scale(wmax);
+    u64 sa = 0;
+    for (int t = tid; t < T; t += nt) sa += to_fixed(weight_of(u[t], p.eps), sw);
+    const u64 SA = block_sum_u64(sa, sm.scratch);
+    const double dSA = (double)SA;
+
+    // ---- EMA credit and the mass used for segmentation
+    u64 sh = 0;
+    if (ema_on) {
+        const float oml = __fsub_rn(1.0f, p.lambda);
+        float cmax = 0.0f;
+        for (int t = tid; t < T; t += nt) {
+            const u64 A = to_fixed(weight_of(u[t], p.eps), sw);
+            const float m = __double2float_rn(__ddiv_rn((double)A, dSA));
+            const float cn = __fadd_rn(__fmul_rn(p.lambda, credit[t]), __fmul_rn(oml, m));
+            credit[t] = cn;
+            if (mass_dbg) mass_dbg[t] = m;
+            cmax = fmaxf(cmax, cn);
+        }
+        cmax = block_max_f32(cmax, sm.scratch);
+        u64 scsum = 0;
+        double scl = 0.0;
+        if (cmax > 0.0f) {
+            scl = fix_scale(cmax);
+            for (int t = tid; t < T; t += nt) scsum += to_fixed(credit[t], scl);
+        }
+        const u64 SC = block_sum_u64(scsum, sm.scratch);
+        const double dSC = (double)SC, bd = (double)p.beta, omb = __dsub_rn(1.0, (double)p.beta);
+        for (int t = tid; t < T; t += nt) {
+            const u64 A = to_fixed(weight_of(u[t], p.eps), sw);
+            const double cur = __dmul_rn(bd, __ddiv_rn((double)A, dSA));
+            double hist_term = 0.0;
+            if (SC > 0) hist_term = __dmul_rn(omb, __ddiv_rn((double)to_fixed(credit[t], scl), dSC));
+            const u64 Hm = (u64)__double2ull_rd(__dmul_rn(__dadd_rn(cur, hist_term), two_f));
+            Cb[t] = Hm;
+            sh += Hm;
+        }
+    } else {
+        for (int t = tid; t < T; t += nt) {
+            const u64 A = to_fixed(weight_of(u[t], p.eps), sw);
+            const double r = __ddiv_rn((double)A, dSA);
+            if (mass_dbg) mass_dbg[t] = __double2float_rn(r);
+            const u64 Hm = (u64)__double2ull_rd(__dmul_rn(r, two_f));
+            Cb[t] = Hm;
+            sh += Hm;
+        }
+    }
+    const u64 SH = block_sum_u64(sh, sm.scratch);
+
+    // ---- inclusive prefix sum and mass-quantile cuts: the token that reaches quantile k
+    //      closes its segment, so the boundary is (position + 1)
+    const u64 S = (u64)p.S;
+    for (int k = tid; k <= p.S; k += nt) raw[k] = T;
+    __syncthreads();
+    u64 carry = 0;
+    for (int base = 0; base < T; base += nt * 4) {
+        const int t0 = base + tid * 4;
+        u64 v[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) v[i] = (t0 + i < T) ? Cb[t0 + i] : 0ull;
+        u64 tot;
+        const u64 exc = carry + block_excl_scan_u64(v[0] + v[1] + v[2] + v[3], sm.scratch, &tot);
+        carry += tot;
+        if (t0 < T) {
+            u64 run = exc;
+            int kprev = quantile_of(exc, S, SH);
+            const int klast = quantile_of(exc + v[0] + v[1] + v[2] + v[3], S, SH);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                if (t0 + i < T) {
+                    run += v[i];
+                    Cb[t0 + i] = run;
+                    if (klast != kprev) {
+                        const int kc = quantile_of(run, S, SH);
+                        for (int k = kprev + 1; k <= kc; ++k) raw[k] = t0 + i + 1;
+                        kprev = kc;
+                    }
+                }
+            }
+        }
+    }
+    __syncthreads();
+
+    // ---- merge short raw segments forward, fold a short tail left, count split pieces
+    if (tid == 0) {
+        int nm = 0;
+        merged[nm++] = 0;
+        int last = 0;
+        for (int k = 1; k < p.S; ++k) {
+            const int e = raw[k];
+            if (e <= last || e >= T) continue;
+            last = e;
+            if (e - merged[nm - 1] >= p.l_min) merged[nm++] = e;
+        }
+        merged[nm++] = T;
+        if (nm > 2 && merged[nm - 1] - merged[nm - 2] < p.l_min) { merged[nm - 2] = T; --nm; }
+        int off = 0;
+        for (int i = 0; i + 1 < nm; ++i) {
+            const int len = merged[i + 1] - merged[i];
+            poff[i] = off;
+            off += (p.l_max > 0 && len > p.l_max) ? (len + p.l_max - 1) / p.l_max : 1;
+        }
+        poff[nm - 1] = off;
+        sm.bcast[0] = nm - 1;
+        sm.bcast[1] = off;
+    }
+    __syncthreads();
+    const int n_merged = sm.bcast[0], n_seg = sm.bcast[1];
+    if (n_seg > sc) { if (tid == 0) set_status(p.status, AMS_ERR_CAPACITY, uid, n_seg, sc); return; }
+    if (tid == 0) bounds[0] = 0;
+    for (int i = 0; i < n_merged; ++i) {
+        const int a = merged[i], len = merged[i + 1] - a, pieces = poff[i + 1] - poff[i];
+        const int bs = len / pieces, extra = len % pieces;
+        for (int j = tid; j < pieces; j += nt) bounds[poff[i] + j + 1] = a + (j + 1) * bs + min(j + 1, extra);
+    }
+    __syncthreads();
+
+    // ---- must-keep sizes and quotas
+    const int ns = max(0, min(p.n_sink, min(p.Tk, T)));
+    const int nl = max(0, min(p.n_last, min(p.Tk - ns, T - ns)));
+    const int Bq = p.Tk - ns - nl;
+    long long smin = 0;
+    for (int i = tid; i < n_seg; i += nt) {
+        const int a = bounds[i], e = bounds[i + 1];
+        Ms[i] = Cb[e - 1] - (a > 0 ? Cb[a - 1] : 0ull);
+        smin += max(0, min(p.q_min, e - a));
+    }
+    smin = block_sum_i64(smin, sm.scratch);
+    const long long Trem = (long long)Bq - smin;
+    long long sq = 0;
+    for (int i = tid; i < n_seg; i += nt) {
+        const int L = bounds[i + 1] - bounds[i];
+        long long qi = max(0, min(p.q_min, L));
+        if (Trem >= 0) qi += (long long)((2ull * (u64)Trem * Ms[i] + SH) / (2ull * SH));
+        if (qi > L) qi = L;
+        quota[i] = (int)qi;
+        sq += qi;
+    }
+    sq = block_sum_i64(sq, sm.scratch);
+    long long Dq = (long long)Bq - sq;
+    if (Dq > 0) {
+        for (int i = tid; i < n_seg; i += nt) cap[i] = bounds[i + 1] - bounds[i] - quota[i];
+        __syncthreads();
+        distribute<true>(Dq, cap, give, Ms, n_seg, sm);
+        for (int i = tid; i < n_seg; i += nt) quota[i] += give[i];
+    } else if (Dq < 0) {
+        for (int i = tid; i < n_seg; i += nt)
+            cap[i] = quota[i] - max(0, min(p.q_min, bounds[i + 1] - bounds[i]));
+        __syncthreads();
+        long long left = distribute<false>(-Dq, cap, give, Ms, n_seg, sm);
+        for (int i = tid; i < n_seg; i += nt) quota[i] -= give[i];
+        if (left > 0) { // the budget cannot cover the minima: go below them
+            __syncthreads();
+            for (int i = tid; i < n_seg; i += nt) cap[i] = quota[i];
+            __syncthreads();
+            distribute<false>(left, cap, give, Ms, n_seg, sm);
+            for (int i = tid; i < n_seg; i += nt) quota[i] -= give[i];
+        }
+    }
+    __syncthreads();
+    if (tid == 0) p.n_seg[uid] = n_seg;
+    for (int i = tid; i < n_seg; i += nt) {
+        p.seg_bounds[(size_t)uid * (sc + 1) + i] = bounds[i];
+        p.quotas[(size_t)uid * sc + i] = quota[i];
+    }
+    if (tid == 0) p.seg_bounds[(size_t)uid * (sc + 1) + n_seg] = T;
+
+    // ---- per-segment top-q_i by (score desc, position asc): one warp per segment
+    int *whist = hist + warp * 256;
+    int *wbc = hist + nw * 256 + warp * 4;
+    for (int s = warp; s < n_seg; s += nw) {
+        const int a = bounds[s], e = bounds[s + 1], q = quota[s], L = e - a;
+        if (q <= 0 || q >= L) {
+            const unsigned char f = q >= L ? 1 : 0;
+            for (int t = a + lane; t < e; t += 32) flags[t] = f;
+            continue;
+        }
+        unsigned thr; int take, ties;
+        radix_select<false>(g, a, e, q, whist, wbc, [](int) { return true; }, &thr, &take, &ties);
+        int seen = 0;
+        for (int base = a; base < e; base += 32) {
+            const int t = base + lane;
+            const unsigned key = t < e ? score_key(g[t]) : 0u;
+            bool keepit = t < e && key > thr;
+            const bool tie = t < e && key == thr;
+            if (take >= ties) keepit |= tie;
+            else {
+                const unsigned bal = __ballot_sync(0xffffffffu, tie);
+                const int rank = seen + __popc(bal & ((1u << lane) - 1u));
+                keepit |= tie && rank < take;
+                seen += __popc(bal);
+            }
+            if (t < e) flags[t] = keepit ? 1 : 0;
+        }
+    }
+    __syncthreads();
+
+    // ---- must-keep prefix and suffix; every must-keep position a segment already chose
+    //      frees one slot, refilled by the best positions not yet kept
+    long long already = 0;
+    for (int i = tid; i < ns + nl; i += nt) {
+        const int t = i < ns ? i : T - nl + (i - ns);
+        already += flags[t];
+        flags[t] = 1;
+    }
+    const int r = (int)block_sum_i64(already, sm.scratch);
+    if (r > 0) {
+        unsigned thr; int take, ties;
+        radix_select<true>(g, 0, T, r, hist, sm.bcast + 4, [flags](int t) { return flags[t] == 0; }, &thr, &take, &ties);
+        int seen = 0;
+        for (int base = 0; base < T; base += nt) {
+            const int t = base + tid;
+            const bool cand = t < T && flags[t] == 0;
+            const unsigned key = cand ? score_key(g[t]) : 0u;
+            bool keepit = cand && key > thr;
+            const bool tie = cand && key == thr;
+            if (take >= ties) keepit |= tie;
+            else {
+                if (seen >= take) { if (keepit) flags[t] = 1; continue; }
+                u64 tot;
+                const int rank = seen + (int)block_excl_scan_u64(tie ? 1ull : 0ull, sm.scratch, &tot);
+                keepit |= tie && rank < take;
+                seen += (int)tot;
+            }
+            if (keepit) flags[t] = 1;
+        }
+    }
+    __syncthreads();
+
+    // ---- ordered compaction of the kept positions
+    int out = 0;
+    for (int base = 0; base < T; base += nt * 16) {
+        const int t0 = base + tid * 16;
+        uint4 f = make_uint4(0, 0, 0, 0);
+        if (t0 < T) f = *reinterpret_cast<const uint4 *>(flags + t0);
+        unsigned wds[4] = {f.x, f.y, f.z, f.w};
+        int cnt = 0;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const bool on = (t0 + i < T) && ((wds[i >> 2] >> ((i & 3) * 8)) & 0xffu);
+            cnt += on;
+        }
+        u64 tot;
+        int pos = out + (int)block_excl_scan_u64((u64)cnt, sm.scratch, &tot);
+        out += (int)tot;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const bool on = (t0 + i < T) && ((wds[i >> 2] >> ((i & 3) * 8)) & 0xffu);
+            if (on) { if (pos < p.Tk) keep[pos] = t0 + i; ++pos; }
+        }
+    }
+    if (out != p.Tk) { if (tid == 0) set_status(p.status, AMS_ERR_INTERNAL, uid, out, p.Tk); return; }
+    __syncthreads();
+
+    // ---- credit rows travel with their tokens; rows beyond the budget start from zero
+    if (ema_on) {
+        float *tmp = reinterpret_cast<float *>(Cb);
+        for (int j = tid; j < p.Tk; j += nt) tmp[j] = credit[keep[j]];
+        __syncthreads();
+        for (int j = tid; j < T; j += nt) credit[j] = j < p.Tk ? tmp[j] : 0.0f;
+    }
+}
+
+int launch_segment_select(const DevParams &p, cudaStream_t s, int *launches)
+{
+    const int units = p.L * p.B * p.H;
+    const int nthreads = 1024;
+    const size_t dyn = (size_t)p.seg_cap * 8 + (size_t)(4 * p.seg_cap + 1) * 4 + (size_t)3 * (p.S + 1) * 4 +
+                       (size_t)(nthreads / 32) * (256 + 4) * 4 + 64;
+    static size_t configured = 0;
+    if (dyn > configured) {
+        if (cudaFuncSetAttribute(k_segment_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
+            return AMS_ERR_CUDA;
+        configured = dyn;
+    }
+    k_segment_select<<<units, nthreads, dyn, s>>>(p);
+    ++*launches;
+    return cudaGetLastError() == cudaSuccess ? AMS_OK : AMS_ERR_CUDA;
+}
+
+} // namespace ams
