@@ -141,6 +141,16 @@ int ams_get_status(ams_state *st, void *stream, int32_t *detail);
 /* Number of kernels the last ams_compress on this handle launched. */
 int32_t ams_last_launch_count(const ams_state *st);
 
+/* Optional per-kernel timing.  With profiling enabled, ams_compress records a CUDA
+ * event on its stream after every kernel it launches (events are host objects; no
+ * device memory is allocated).  ams_get_kernel_times waits for the last call's final
+ * event and writes AMS_KERNEL_SLOTS durations in milliseconds, one per kernel slot
+ * named by ams_kernel_name (a slot launched more than once holds the sum). */
+#define AMS_KERNEL_SLOTS 6
+int ams_set_profiling(ams_state *st, int enable);
+int ams_get_kernel_times(ams_state *st, float *ms);
+const char *ams_kernel_name(int32_t idx);
+
 /* Releases the host handle only. */
 int ams_free(ams_state *st);
 

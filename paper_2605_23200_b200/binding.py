@@ -24,7 +24,8 @@ AMS_SCORER_TOVA, AMS_SCORER_KEYDIFF, AMS_SCORER_EXTERNAL = 0, 1, 2
 
 EXPORTS = ["ams_config_default", "ams_ema_state_bytes", "ams_workspace_bytes", "ams_segment_capacity",
            "ams_init_state", "ams_compress", "ams_get_status", "ams_last_launch_count", "ams_free",
-           "ams_strerror"]
+           "ams_strerror", "ams_set_profiling", "ams_get_kernel_times", "ams_kernel_name"]
+KERNEL_SLOTS = 6
 
 
 class AmsConfig(ctypes.Structure):
@@ -71,6 +72,12 @@ def lib() -> ctypes.CDLL:
         L.ams_last_launch_count.restype = ctypes.c_int32
         L.ams_free.argtypes = [ctypes.c_void_p]
         L.ams_free.restype = ctypes.c_int
+        L.ams_set_profiling.argtypes = [ctypes.c_void_p, ctypes.c_int]
+        L.ams_set_profiling.restype = ctypes.c_int
+        L.ams_get_kernel_times.argtypes = [ctypes.c_void_p, ctypes.POINTER(ctypes.c_float)]
+        L.ams_get_kernel_times.restype = ctypes.c_int
+        L.ams_kernel_name.argtypes = [ctypes.c_int32]
+        L.ams_kernel_name.restype = ctypes.c_char_p
         L.ams_strerror.argtypes = [ctypes.c_int]
         L.ams_strerror.restype = ctypes.c_char_p
         _lib = L
@@ -178,6 +185,19 @@ class AmsCompressor:
         if check and rc != AMS_OK:
             raise AmsError(rc, "device status", list(detail))
         return rc, list(detail)
+
+    def set_profiling(self, enable: bool) -> None:
+        rc = lib().ams_set_profiling(self._h, 1 if enable else 0)
+        if rc != AMS_OK:
+            raise AmsError(rc, "ams_set_profiling")
+
+    def kernel_times_ms(self) -> dict:
+        """Per-kernel durations of the last call (profiling must be on); waits for the call to finish."""
+        buf = (ctypes.c_float * KERNEL_SLOTS)()
+        rc = lib().ams_get_kernel_times(self._h, buf)
+        if rc != AMS_OK:
+            raise AmsError(rc, "ams_get_kernel_times")
+        return {lib().ams_kernel_name(i).decode(): float(buf[i]) for i in range(KERNEL_SLOTS)}
 
     @property
     def last_launch_count(self) -> int:

@@ -93,6 +93,10 @@ struct ams_state {
     unsigned char *ws;
     void *ema;
     int32_t last_launches;
+    cudaEvent_t ev[32];
+    bool profiling;
+    int n_ev;
+    int ev_ids[32];
 };
 
 extern "C" {
@@ -156,6 +160,8 @@ int ams_init_state(const ams_config *cfg, void *ema_state, void *workspace, size
     st->ws = (unsigned char *)workspace;
     st->ema = ema_state;
     st->last_launches = 0;
+    st->profiling = false;
+    st->n_ev = 0;
     *out = st;
     return AMS_OK;
 }
@@ -206,10 +212,15 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
     p.rows_pad = scorer_id == AMS_SCORER_TOVA ? rows_padded(p.rows) : kHeadDim;
     p.status = (int *)(st->ws + y.status);
 
-    int launches = 0, rc = AMS_OK;
-    if (scorer_id == AMS_SCORER_TOVA) rc = launch_score_tova(p, s, &launches);
-    else if (scorer_id == AMS_SCORER_KEYDIFF) rc = launch_score_keydiff(p, s, &launches);
-    if (rc == AMS_OK) rc = launch_segment_select(p, s, &launches);
+    int rc = AMS_OK;
+    LaunchCtx ctx;
+    ctx.s = s;
+    ctx.ev = st->profiling ? st->ev : nullptr;
+    ctx.max_ev = 32;
+    ctx.begin();
+    if (scorer_id == AMS_SCORER_TOVA) rc = launch_score_tova(p, ctx);
+    else if (scorer_id == AMS_SCORER_KEYDIFF) rc = launch_score_keydiff(p, ctx);
+    if (rc == AMS_OK) rc = launch_segment_select(p, ctx);
     if (rc == AMS_OK && dbg) {
         // inspection copies are taken before the table is rewritten
         const size_t U = (size_t)p.L * p.B * p.H;
@@ -221,8 +232,10 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
         if (dbg->keep_idx && e == cudaSuccess) e = cudaMemcpyAsync(dbg->keep_idx, p.keep_idx, U * (size_t)p.Tk * 4, cudaMemcpyDeviceToDevice, s);
         if (e != cudaSuccess) rc = AMS_ERR_CUDA;
     }
-    if (rc == AMS_OK) rc = launch_gather(p, s, &launches);
-    st->last_launches = launches;
+    if (rc == AMS_OK) rc = launch_gather(p, ctx);
+    st->last_launches = ctx.launches;
+    st->n_ev = ctx.n_ev;
+    memcpy(st->ev_ids, ctx.ids, sizeof ctx.ids);
     return rc;
 }
 
@@ -240,9 +253,47 @@ int ams_get_status(ams_state *st, void *stream, int32_t *detail)
 
 int32_t ams_last_launch_count(const ams_state *st) { return st ? st->last_launches : 0; }
 
+int ams_set_profiling(ams_state *st, int enable)
+{
+    if (!st) return AMS_ERR_INVALID_ARG;
+    if (enable && !st->profiling) {
+        for (int i = 0; i < 32; ++i)
+            if (cudaEventCreate(&st->ev[i]) != cudaSuccess) return AMS_ERR_CUDA;
+        st->profiling = true;
+    } else if (!enable && st->profiling) {
+        for (int i = 0; i < 32; ++i) cudaEventDestroy(st->ev[i]);
+        st->profiling = false;
+    }
+    st->n_ev = 0;
+    return AMS_OK;
+}
+
+int ams_get_kernel_times(ams_state *st, float *ms)
+{
+    if (!st || !ms) return AMS_ERR_INVALID_ARG;
+    for (int i = 0; i < kKernCount; ++i) ms[i] = 0.0f;
+    if (!st->profiling || st->n_ev < 2) return AMS_ERR_INVALID_ARG;
+    if (cudaEventSynchronize(st->ev[st->n_ev - 1]) != cudaSuccess) return AMS_ERR_CUDA;
+    for (int i = 1; i < st->n_ev; ++i) {
+        float t = 0.0f;
+        if (cudaEventElapsedTime(&t, st->ev[i - 1], st->ev[i]) != cudaSuccess) return AMS_ERR_CUDA;
+        const int id = st->ev_ids[i];
+        if (id >= 0 && id < kKernCount) ms[id] += t;
+    }
+    return AMS_OK;
+}
+
+const char *ams_kernel_name(int32_t idx)
+{
+    static const char *names[kKernCount] = {"score_phase1", "score_combine", "score_phase2", "segment_select",
+                                            "gather", "table_update"};
+    return idx >= 0 && idx < kKernCount ? names[idx] : nullptr;
+}
+
 int ams_free(ams_state *st)
 {
     if (!st) return AMS_ERR_INVALID_ARG;
+    if (st->profiling) ams_set_profiling(st, 0);
     delete st;
     return AMS_OK;
 }

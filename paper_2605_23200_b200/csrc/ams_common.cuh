@@ -167,9 +167,31 @@ __device__ __forceinline__ uint4 ld_stream16(const void *ptr)
 
 // Host-side launchers (one per translation unit).
 int tova_rows_block(int rows); // query rows handled per pass of the TOVA kernel (8..128)
-int launch_score_tova(const DevParams &p, cudaStream_t s, int *launches);
-int launch_score_keydiff(const DevParams &p, cudaStream_t s, int *launches);
-int launch_segment_select(const DevParams &p, cudaStream_t s, int *launches);
-int launch_gather(const DevParams &p, cudaStream_t s, int *launches);
+enum KernelId { kKernScore1 = 0, kKernScoreCombine, kKernScore2, kKernSegmentSelect, kKernGather, kKernTable, kKernCount };
+
+// Stream, launch counter and optional per-kernel timing events of one ams_compress call.
+struct LaunchCtx {
+    cudaStream_t s;
+    int launches;
+    cudaEvent_t *ev; // null unless profiling; ev[0] is recorded before the first launch
+    int n_ev, max_ev;
+    int ids[32];
+    void begin()
+    {
+        launches = 0;
+        n_ev = 0;
+        if (ev) { cudaEventRecord(ev[0], s); n_ev = 1; }
+    }
+    void mark(int id) // call right after a launch
+    {
+        ++launches;
+        if (ev && n_ev < max_ev) { cudaEventRecord(ev[n_ev], s); ids[n_ev] = id; ++n_ev; }
+    }
+};
+
+int launch_score_tova(const DevParams &p, LaunchCtx &ctx);
+int launch_score_keydiff(const DevParams &p, LaunchCtx &ctx);
+int launch_segment_select(const DevParams &p, LaunchCtx &ctx);
+int launch_gather(const DevParams &p, LaunchCtx &ctx);
 
 } // namespace ams

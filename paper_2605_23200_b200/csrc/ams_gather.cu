@@ -74,14 +74,14 @@ __global__ void k_table_update(DevParams p)
 
 } // namespace
 
-int launch_gather(const DevParams &p, cudaStream_t s, int *launches)
+int launch_gather(const DevParams &p, LaunchCtx &ctx)
 {
     const int n_rows = p.Tk * p.H;
     dim3 grid((n_rows + kRowsPerBlock - 1) / kRowsPerBlock, p.L * p.B);
-    k_gather<<<grid, kGatherThreads, 0, s>>>(p);
-    ++*launches;
-    k_table_update<<<p.B, 128, 0, s>>>(p);
-    ++*launches;
+    k_gather<<<grid, kGatherThreads, 0, ctx.s>>>(p);
+    ctx.mark(kKernGather);
+    k_table_update<<<p.B, 128, 0, ctx.s>>>(p);
+    ctx.mark(kKernTable);
     return cudaGetLastError() == cudaSuccess ? AMS_OK : AMS_ERR_CUDA;
 }
 

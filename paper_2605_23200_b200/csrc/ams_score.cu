@@ -322,13 +322,15 @@ __global__ void __launch_bounds__(kKdThreads) k_keydiff_score(DevParams p)
 }
 
 template <int NTB>
-void launch_tova_ntb(const DevParams &p, cudaStream_t s, int *launches)
+void launch_tova_ntb(const DevParams &p, LaunchCtx &ctx)
 {
     const dim3 grid(p.n_slices, p.L * p.B * p.H);
-    k_tova<NTB, 1><<<grid, kTovaThreads, 0, s>>>(p);
-    k_tova_combine<<<p.L * p.B * p.H, 128, 0, s>>>(p);
-    k_tova<NTB, 2><<<grid, kTovaThreads, 0, s>>>(p);
-    *launches += 3;
+    k_tova<NTB, 1><<<grid, kTovaThreads, 0, ctx.s>>>(p);
+    ctx.mark(kKernScore1);
+    k_tova_combine<<<p.L * p.B * p.H, 128, 0, ctx.s>>>(p);
+    ctx.mark(kKernScoreCombine);
+    k_tova<NTB, 2><<<grid, kTovaThreads, 0, ctx.s>>>(p);
+    ctx.mark(kKernScore2);
 }
 
 } // namespace
@@ -340,25 +342,27 @@ int tova_rows_block(int rows)
     return ntb * 8;
 }
 
-int launch_score_tova(const DevParams &p, cudaStream_t s, int *launches)
+int launch_score_tova(const DevParams &p, LaunchCtx &ctx)
 {
     switch (tova_rows_block(p.rows) / 8) {
-    case 1: launch_tova_ntb<1>(p, s, launches); break;
-    case 2: launch_tova_ntb<2>(p, s, launches); break;
-    case 4: launch_tova_ntb<4>(p, s, launches); break;
-    case 8: launch_tova_ntb<8>(p, s, launches); break;
-    default: launch_tova_ntb<16>(p, s, launches); break;
+    case 1: launch_tova_ntb<1>(p, ctx); break;
+    case 2: launch_tova_ntb<2>(p, ctx); break;
+    case 4: launch_tova_ntb<4>(p, ctx); break;
+    case 8: launch_tova_ntb<8>(p, ctx); break;
+    default: launch_tova_ntb<16>(p, ctx); break;
     }
     return cudaGetLastError() == cudaSuccess ? AMS_OK : AMS_ERR_CUDA;
 }
 
-int launch_score_keydiff(const DevParams &p, cudaStream_t s, int *launches)
+int launch_score_keydiff(const DevParams &p, LaunchCtx &ctx)
 {
     const dim3 grid(p.n_slices, p.L * p.B * p.H);
-    k_keydiff_sum<<<grid, kKdThreads, 0, s>>>(p);
-    k_keydiff_combine<<<p.L * p.B * p.H, kHeadDim, 0, s>>>(p);
-    k_keydiff_score<<<grid, kKdThreads, 0, s>>>(p);
-    *launches += 3;
+    k_keydiff_sum<<<grid, kKdThreads, 0, ctx.s>>>(p);
+    ctx.mark(kKernScore1);
+    k_keydiff_combine<<<p.L * p.B * p.H, kHeadDim, 0, ctx.s>>>(p);
+    ctx.mark(kKernScoreCombine);
+    k_keydiff_score<<<grid, kKdThreads, 0, ctx.s>>>(p);
+    ctx.mark(kKernScore2);
     return cudaGetLastError() == cudaSuccess ? AMS_OK : AMS_ERR_CUDA;
 }
 

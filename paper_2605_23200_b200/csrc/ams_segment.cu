@@ -473,7 +473,7 @@ __global__ void __launch_bounds__(1024) k_segment_select(DevParams p)
     }
 }
 
-int launch_segment_select(const DevParams &p, cudaStream_t s, int *launches)
+int launch_segment_select(const DevParams &p, LaunchCtx &ctx)
 {
     const int units = p.L * p.B * p.H;
     const int nthreads = 1024;
@@ -485,8 +485,8 @@ int launch_segment_select(const DevParams &p, cudaStream_t s, int *launches)
             return AMS_ERR_CUDA;
         configured = dyn;
     }
-    k_segment_select<<<units, nthreads, dyn, s>>>(p);
-    ++*launches;
+    k_segment_select<<<units, nthreads, dyn, ctx.s>>>(p);
+    ctx.mark(kKernSegmentSelect);
     return cudaGetLastError() == cudaSuccess ? AMS_OK : AMS_ERR_CUDA;
 }
 
