@@ -129,6 +129,8 @@ def run_ours(args, rank, world, local_rank):
         barrier()
     binding.lib()
     wl = inputs.CONFIGS[args.config]
+    if args.layers:
+        wl = wl.scaled(n_layers=args.layers, resident_layers=0, name=wl.name + f"_REDUCED_to_{args.layers}_layers")
     cache = inputs.make_cache(wl, dev)
     comp = binding.AmsCompressor(binding.config_for(wl), dev)
     stream = torch.cuda.current_stream(dev)
@@ -202,17 +204,19 @@ def run_ours(args, rank, world, local_rank):
         comp.status()  # reads the device status word and synchronises the stream
 
     n_e2e = min(args.steps, 50)
-    for _ in range(3):
-        comp.ema_state.zero_()
-        e2e_step()
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(n_e2e):
-        comp.ema_state.zero_()
-        e2e_step()
-    torch.cuda.synchronize(dev)
-    e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3, dev)
-    assert int(out_lens[0]) == wl.budget
+    e2e_ms = None
+    if not args.no_e2e:
+        for _ in range(3):
+            comp.ema_state.zero_()
+            e2e_step()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            comp.ema_state.zero_()
+            e2e_step()
+        torch.cuda.synchronize(dev)
+        e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3, dev)
+        assert int(out_lens[0]) == wl.budget
 
     k_read, moved = algorithmic_bytes(wl, lens0.cpu().numpy())
     peak, peak_kind = _peaks()
@@ -239,8 +243,8 @@ def run_ours(args, rank, world, local_rank):
         "roofline": {"kernel": dominant, "bound": "hbm", "achieved": dom_bytes / (dom_ms * 1e-3) / 1e9, "peak": peak,
                      "peak_kind": peak_kind, "unit": "GB/s", "frac": dom_bytes / (dom_ms * 1e-3) / 1e9 / peak,
                      "traffic": None, "algorithmic_bytes_per_launch": dom_bytes},
-        "e2e": {"value": world * n_e2e / (e2e_ms / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "steps": n_e2e},
+        "e2e": None if e2e_ms is None else {"value": world * n_e2e / (e2e_ms / 1e3), "unit": UNIT,
+                                            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e},
         "clocks": clocks,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -341,6 +345,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=1)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="profiling only: run a reduced layer count")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
