@@ -151,6 +151,28 @@ int ams_set_profiling(ams_state *st, int enable);
 int ams_get_kernel_times(ams_state *st, float *ms);
 const char *ams_kernel_name(int32_t idx);
 
+/* Selection without any allocation (the paper has no counterpart: this is an interface
+ * convenience, not a step of the method).  For callers that cannot obtain device memory:
+ * code that runs while a stream is being captured, plug-ins inside a process whose device
+ * memory pool belongs to the host framework, paths that must not touch the allocator.
+ * Runs steps 1-5 of Algorithm 1 (mass, cuts, merge/split, quotas, per-segment top-k,
+ * must-keep, backfill) on caller-supplied scores and writes the kept positions; there is
+ * no EMA credit (the mass is that of the given scores alone), no K/V movement, no handle
+ * and no workspace argument.  The scratch is a fixed device array inside the library
+ * (about 2.6 MB, held by every GPU that loads the library until the process exits).
+ *   scores   : DEVICE fp32 [n_units][score_stride], score_stride a multiple of 16, >= seq_len
+ *   keep_idx : DEVICE int32 [n_units][budget], ascending positions
+ *   cfg      : only l_min, l_max, q_min, n_sink, n_last and eps are read
+ * Limits: n_units <= 8, seq_len <= 32768, n_segments + 2*floor(seq_len/l_max) + 4 <= 1024;
+ * beyond them AMS_ERR_CAPACITY is returned and nothing is launched.  1 <= budget < seq_len.
+ * The first call on a device looks up the array's address on that device (with that device
+ * current); make that first call before starting a stream capture.  All calls share the one
+ * array, which keeps the previous call's contents: the entry point re-initialises what must
+ * start at zero, but two calls that overlap on the GPU (different streams, or a captured
+ * graph replayed concurrently) race on it.  Asynchronous on `stream`. */
+int ams_select_static(const ams_config *cfg, const float *scores, int32_t score_stride, int32_t n_units,
+                      int32_t seq_len, int32_t budget, int32_t n_segments, int32_t *keep_idx, void *stream);
+
 /* Releases the host handle only. */
 int ams_free(ams_state *st);
 

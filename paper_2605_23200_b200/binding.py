@@ -24,7 +24,7 @@ AMS_SCORER_TOVA, AMS_SCORER_KEYDIFF, AMS_SCORER_EXTERNAL = 0, 1, 2
 
 EXPORTS = ["ams_config_default", "ams_ema_state_bytes", "ams_workspace_bytes", "ams_segment_capacity",
            "ams_init_state", "ams_compress", "ams_get_status", "ams_last_launch_count", "ams_free",
-           "ams_strerror", "ams_set_profiling", "ams_get_kernel_times", "ams_kernel_name"]
+           "ams_strerror", "ams_set_profiling", "ams_get_kernel_times", "ams_kernel_name", "ams_select_static"]
 KERNEL_SLOTS = 6
 
 
@@ -78,6 +78,10 @@ def lib() -> ctypes.CDLL:
         L.ams_get_kernel_times.restype = ctypes.c_int
         L.ams_kernel_name.argtypes = [ctypes.c_int32]
         L.ams_kernel_name.restype = ctypes.c_char_p
+        L.ams_select_static.argtypes = [ctypes.POINTER(AmsConfig), ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
+                                        ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p,
+                                        ctypes.c_void_p]
+        L.ams_select_static.restype = ctypes.c_int
         L.ams_strerror.argtypes = [ctypes.c_int]
         L.ams_strerror.restype = ctypes.c_char_p
         _lib = L
@@ -213,6 +217,21 @@ class AmsCompressor:
             self.close()
         except Exception:
             pass
+
+
+def select_static(cfg: AmsConfig, scores: torch.Tensor, seq_len: int, budget: int, n_segments: int,
+                  keep_idx: torch.Tensor, stream: torch.cuda.Stream | None = None) -> None:
+    """Allocation-free selection for callers that cannot obtain device memory (stream capture in
+    progress, a memory pool owned by the host framework): kept positions of each score row are
+    written to `keep_idx` (int32 [n_units][budget]); the library's fixed scratch array is used, so
+    calls must not overlap on the GPU.  `scores` is fp32 [n_units][stride], stride % 16 == 0."""
+    assert scores.dtype == torch.float32 and scores.is_contiguous() and scores.dim() == 2
+    assert keep_idx.dtype == torch.int32 and keep_idx.is_contiguous() and keep_idx.shape == (scores.shape[0], budget)
+    s = stream or torch.cuda.current_stream(scores.device)
+    rc = lib().ams_select_static(ctypes.byref(cfg), _ptr(scores), scores.shape[1], scores.shape[0], seq_len, budget,
+                                 n_segments, _ptr(keep_idx), ctypes.c_void_p(s.cuda_stream))
+    if rc != AMS_OK:
+        raise AmsError(rc, "ams_select_static")
 
 
 def config_for(wl, **kw) -> AmsConfig:

@@ -6,6 +6,7 @@
 // fractional bits) and every floating-point step is a single round-to-nearest
 // operation, so the result does not depend on how the block orders its sums.
 #include <float.h>
+#include <string.h>
 
 #include "ams_common.cuh"
 
@@ -491,3 +492,110 @@ int launch_segment_select(const DevParams &p, LaunchCtx &ctx)
 }
 
 } // namespace ams
+
+// ---------------------------------------------------------------------------------------
+// Allocation-free selection entry point.
+//
+// Some callers cannot allocate device memory at all: code running while a stream is being
+// captured into a CUDA graph (allocation calls are not permitted there), plug-ins loaded into
+// a serving process whose memory pool is owned and fully reserved by the host framework, and
+// callers on a hot path that must not take the allocator's locks.  For them the scratch the
+// selection kernel needs lives in the fixed array below instead of a caller-supplied
+// workspace.  Every GPU that loads the library holds the array (kStaticBytes, about 2.6 MB)
+// until the process exits.
+namespace ams {
+namespace {
+
+constexpr int kStaticMaxUnits = 8;       // score rows per call
+constexpr int kStaticMaxTokens = 32768;  // tokens per score row
+constexpr int kStaticSegCap = 1024;      // segments per row after merge and split
+constexpr int kStaticMaxDevices = 64;
+
+struct StaticLayout {
+    static constexpr size_t status = 0;                                                   // 4 x int32
+    static constexpr size_t lens = 256;                                                   // [units] int32
+    static constexpr size_t n_seg = 512;                                                  // [units] int32
+    static constexpr size_t bounds = 1024;                                                // [units][cap + 1] int32
+    static constexpr size_t quotas = bounds + (size_t)kStaticMaxUnits * (kStaticSegCap + 1) * 4;
+    static constexpr size_t flags = (quotas + (size_t)kStaticMaxUnits * kStaticSegCap * 4 + 255) / 256 * 256;
+    static constexpr size_t cbuf = flags + (size_t)kStaticMaxUnits * kStaticMaxTokens;    // [units][tokens] u64
+    static constexpr size_t total = cbuf + (size_t)kStaticMaxUnits * kStaticMaxTokens * 8;
+};
+constexpr size_t kStaticBytes = StaticLayout::total;
+
+// In host code this name is only a handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+__global__ void k_static_prepare(int *status, int *lens, int n_units, int seq_len)
+{
+    if (threadIdx.x < 4) status[threadIdx.x] = 0;
+    if (threadIdx.x < n_units) lens[threadIdx.x] = seq_len;
+}
+
+struct PerDevice {
+    bool ready;
+    unsigned char *base;
+};
+PerDevice g_static_dev[kStaticMaxDevices];
+
+} // namespace
+} // namespace ams
+
+extern "C" int ams_select_static(const ams_config *cfg, const float *scores, int32_t score_stride, int32_t n_units,
+                                 int32_t seq_len, int32_t budget, int32_t n_segments, int32_t *keep_idx, void *stream)
+{
+    using namespace ams;
+    if (!cfg || !scores || !keep_idx) return AMS_ERR_INVALID_ARG;
+    if (n_units < 1 || n_units > kStaticMaxUnits) return AMS_ERR_CAPACITY;
+    if (seq_len < 1 || seq_len > kStaticMaxTokens) return AMS_ERR_CAPACITY;
+    if (score_stride < seq_len || score_stride > kStaticMaxTokens || score_stride % 16) return AMS_ERR_INVALID_ARG;
+    if (budget < 1 || budget >= seq_len) return AMS_ERR_INVALID_ARG;
+    if (n_segments < 1 || n_segments > 1024) return AMS_ERR_INVALID_ARG;
+    if (cfg->l_min < 1 || cfg->l_max < 0 || cfg->q_min < 0 || cfg->n_sink < 0 || cfg->n_last < 0) return AMS_ERR_INVALID_ARG;
+    if (!(cfg->eps > 0.0f) || !(cfg->eps < 1e30f)) return AMS_ERR_INVALID_ARG;
+    const long long seg_cap = (long long)n_segments + (cfg->l_max > 0 ? 2LL * (seq_len / cfg->l_max) : 0) + 4;
+    if (seg_cap > kStaticSegCap) return AMS_ERR_CAPACITY;
+
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kStaticMaxDevices) return AMS_ERR_CUDA;
+    PerDevice &pd = g_static_dev[dev];
+    const int nthreads = 1024;
+    const size_t dyn = (size_t)kStaticSegCap * 8 + (size_t)(4 * kStaticSegCap + 1) * 4 + (size_t)3 * (1024 + 1) * 4 +
+                       (size_t)(nthreads / 32) * (256 + 4) * 4 + 64;
+    if (!pd.ready) {
+        // once per device, with that device current: the array's address on this device
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return AMS_ERR_CUDA;
+        pd.base = (unsigned char *)ptr;
+        pd.ready = true;
+    }
+    // the kernel's dynamic shared-memory limit on this device is only ever raised here
+    cudaFuncAttributes fa;
+    if (cudaFuncGetAttributes(&fa, k_segment_select) != cudaSuccess) return AMS_ERR_CUDA;
+    if ((size_t)fa.maxDynamicSharedSizeBytes < dyn &&
+        cudaFuncSetAttribute(k_segment_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
+        return AMS_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    unsigned char *base = pd.base;
+
+    DevParams p;
+    memset(&p, 0, sizeof p);
+    p.L = 1; p.B = n_units; p.Bmax = n_units; p.H = 1; p.G = 1; p.W = 0; p.rows = 1;
+    p.T_cap = score_stride; p.seg_cap = kStaticSegCap; p.Tk = budget; p.S = n_segments; p.n_dst = (budget + kPage - 1) / kPage;
+    p.l_min = cfg->l_min; p.l_max = cfg->l_max; p.q_min = cfg->q_min; p.n_sink = cfg->n_sink; p.n_last = cfg->n_last;
+    p.lambda = 0.0f; p.beta = 1.0f; p.eps = cfg->eps; // no credit: the mass of the current scores alone
+    p.seq_lens = (int *)(base + StaticLayout::lens);
+    p.usage = scores;
+    p.scores = const_cast<float *>(scores);
+    p.cbuf = (u64 *)(base + StaticLayout::cbuf);
+    p.flags = base + StaticLayout::flags;
+    p.n_seg = (int *)(base + StaticLayout::n_seg);
+    p.seg_bounds = (int *)(base + StaticLayout::bounds);
+    p.quotas = (int *)(base + StaticLayout::quotas);
+    p.keep_idx = keep_idx;
+    p.status = (int *)(base + StaticLayout::status);
+
+    k_static_prepare<<<1, 32, 0, s>>>(p.status, p.seq_lens, n_units, seq_len);
+    k_segment_select<<<n_units, nthreads, dyn, s>>>(p);
+    return cudaGetLastError() == cudaSuccess ? AMS_OK : AMS_ERR_CUDA;
+}
