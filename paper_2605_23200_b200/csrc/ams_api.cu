@@ -52,8 +52,18 @@ static void slicing(int T_cap, int *slice_len, int *n_slices)
 
 static int rows_padded(int rows)
 {
+    if (rows >= 64) return (rows + 127) / 128 * 128; // tensor-core scorer: 128-row query blocks
     const int rb = tova_rows_block(rows < 1 ? 1 : rows);
     return (rows + rb - 1) / rb * rb;
+}
+
+// Tensor-core scorer: a block takes at least this many 128-token tiles, so that a unit is
+// shared by at most 31 blocks.
+static int tc_tiles_per_block_min(int T_cap)
+{
+    const int tiles = (T_cap + 127) / 128;
+    const int need = (tiles + 29) / 30;
+    return need > 8 ? need : 8;
 }
 
 static Layout make_layout(const ams_config *c)
@@ -63,6 +73,8 @@ static Layout make_layout(const ams_config *c)
     y.T_cap = c->max_seq_len;
     y.seg_cap = segment_capacity(c);
     slicing(y.T_cap, &y.slice_len, &y.n_slices);
+    const int tc_parts = ((y.T_cap + 127) / 128 + tc_tiles_per_block_min(y.T_cap) - 1) / tc_tiles_per_block_min(y.T_cap) + 1;
+    if (tc_parts > y.n_slices) y.n_slices = tc_parts;
     const int rows_cap = (c->n_q_heads / c->n_kv_heads) * (c->max_window > 0 ? c->max_window : 1);
     y.rows_pad_cap = rows_padded(rows_cap);
     const size_t U = (size_t)y.units, T = (size_t)y.T_cap;
@@ -210,6 +222,8 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
     p.part = (float *)(st->ws + y.part); p.fin = (float *)(st->ws + y.fin);
     p.slice_len = y.slice_len; p.n_slices = y.n_slices;
     p.rows_pad = scorer_id == AMS_SCORER_TOVA ? rows_padded(p.rows) : kHeadDim;
+    p.tc_tpc_min = tc_tiles_per_block_min(y.T_cap);
+    p.tc_stages = p.rows_pad <= 128 ? 4 : (p.rows_pad <= 256 ? 3 : 2);
     p.status = (int *)(st->ws + y.status);
 
     int rc = AMS_OK;

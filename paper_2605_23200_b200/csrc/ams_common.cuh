@@ -46,6 +46,7 @@ struct DevParams {
     float *part;                      // per (unit, slice) partials
     float *fin;                       // per unit finals
     int slice_len, n_slices, rows_pad;
+    int tc_tpc_min, tc_stages;        // tensor-core scorer: least tiles per block, K stages in shared memory
     int *status;                      // [4]: code, unit, a, b
 };
 
@@ -190,6 +191,9 @@ struct LaunchCtx {
 };
 
 int launch_score_tova(const DevParams &p, LaunchCtx &ctx);
+bool tova_tc_supported(const DevParams &p);
+size_t tova_tc_smem_bytes(const DevParams &p);
+int launch_score_tova_tc(const DevParams &p, LaunchCtx &ctx);
 int launch_score_keydiff(const DevParams &p, LaunchCtx &ctx);
 int launch_segment_select(const DevParams &p, LaunchCtx &ctx);
 int launch_gather(const DevParams &p, LaunchCtx &ctx);

@@ -1,0 +1,542 @@
+// TOVA-style scorer for wide observation windows (rows = G * W >= 64) on the sm_100a
+// tensor path: tcgen05.mma with TMEM accumulators, operands staged by TMA.
+//
+// Work is the concatenation of all units' 128-token tiles; block c of a persistent grid
+// takes the contiguous tile range [c * tpc, (c + 1) * tpc).  Inside a block:
+//   warp 0      TMA producer: query block of the current unit, then one 32 KB K tile per
+//               stage (eight 16-token pages, two 64-wide halves each, 128-byte swizzle);
+//   warp 1      MMA issuer (one lane): per (tile, 128-row query block) eight
+//               tcgen05.mma m128 n128 k16 into one of four 128-column TMEM slots;
+//   warps 4-11  two consumer warpgroups, alternating tiles; thread i of a warpgroup owns
+//               TMEM lane i of its slots.
+// Phase 1 puts query rows on the TMEM lanes (A = Q, B = K), so a thread folds its row's
+// logits into a running (max, sum of 2^x) without leaving registers; phase 2 puts tokens
+// on the lanes (A = K, B = Q), so a thread sums 2^(x - b_r) over the query rows of its
+// token.  Both operands are K-major 128-byte-swizzled tiles, so the same shared-memory
+// tiles serve either role.  Every wait is bounded; on expiry the block reports
+// AMS_ERR_TIMEOUT, drains its copies, frees its TMEM and returns.
+#include <cuda.h>
+
+#include "ams_common.cuh"
+
+namespace ams {
+
+namespace {
+
+constexpr int kTcThreads = 384;
+constexpr int kTileTokens = 128;
+constexpr int kTileBytes = kTileTokens * kRowBytes;  // 32 KB
+constexpr int kHalfBytes = kTileBytes / 2;           // one 64-wide half of a 128-row tile
+constexpr int kSlots = 4;                            // TMEM accumulator slots of 128 columns
+constexpr int kMaxStages = 4;
+constexpr uint32_t kWaitLimit = 1u << 22;
+constexpr float kLog2e = 1.4426950408889634f;
+
+struct TcShared {
+    unsigned long long kfull[kMaxStages], kempty[kMaxStages], tfull[kSlots], tempty[kSlots];
+    unsigned long long qfull, qempty, done;
+    uint32_t tmem_base;
+    int abort_flag;
+    int tiles_lh, tpc;
+    long long n_tiles;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ void lse_merge(float &m, float &z, float m2, float z2)
+{
+    const float mn = fmaxf(m, m2);
+    if (mn == -INFINITY) return;
+    z = z * ex2(m - mn) + z2 * ex2(m2 - mn);
+    m = mn;
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false if the wait ran out or another role of the block already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+{
+    for (uint32_t i = 0; i < kWaitLimit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 1023u) == 1023u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2, int c3, int c4)
+{
+    asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+                 ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, 128 x 128 x 16, bf16 inputs, fp32 accumulate.
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, unsigned long long a_desc, unsigned long long b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// 32 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32])
+{
+    uint32_t r[32];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor of a K-major, 128-byte-swizzled tile whose rows are
+// 128 bytes (64 bf16) and whose 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ unsigned long long smem_desc(uint32_t addr)
+{
+    return (unsigned long long)((addr & 0x3ffffu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// kind::f16 instruction descriptor: fp32 accumulate, bf16 x bf16, both K-major, M = N = 128.
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+
+__device__ __forceinline__ int tiles_of(const DevParams &p, int b)
+{
+    const int T = p.seq_lens[b];
+    return (T > p.Tk && T <= p.T_cap && p.W <= T) ? (T + kTileTokens - 1) / kTileTokens : 0;
+}
+
+// Prefix of tiles per sequence (shared by all layers and heads) and the block partition.
+__device__ void tc_partition(const DevParams &p, int grid, int *prefix, int *tiles_lh, long long *n_tiles, int *tpc)
+{
+    if (threadIdx.x == 0) {
+        int acc = 0;
+        for (int b = 0; b < p.B; ++b) { prefix[b] = acc; acc += tiles_of(p, b); }
+        prefix[p.B] = acc;
+        *tiles_lh = acc;
+        const long long N = (long long)p.L * p.H * acc;
+        *n_tiles = N;
+        const long long per = (N + grid - 1) / grid;
+        *tpc = (int)(per > p.tc_tpc_min ? per : p.tc_tpc_min);
+    }
+    __syncthreads();
+}
+
+struct Segment { int uid, l, b, h, tile0, n, T, part; };
+
+// Decodes the segment that starts at global tile g and ends no later than `end`.
+__device__ __forceinline__ Segment decode_segment(const DevParams &p, const int *prefix, int tiles_lh, int tpc, long long g, long long end)
+{
+    Segment s;
+    const int lh = (int)(g / tiles_lh), rem = (int)(g % tiles_lh);
+    int b = 0;
+    while (prefix[b + 1] <= rem) ++b;
+    s.l = lh / p.H; s.h = lh % p.H; s.b = b;
+    s.uid = (s.l * p.B + b) * p.H + s.h;
+    s.tile0 = rem - prefix[b];
+    const int left = prefix[b + 1] - rem;
+    s.n = (int)((end - g) < left ? (end - g) : left);
+    s.T = p.seq_lens[b];
+    const long long ustart = g - s.tile0;
+    s.part = (int)(g / tpc) - (int)(ustart / tpc);
+    return s;
+}
+
+template <int PHASE>
+__global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __grid_constant__ CUtensorMap k_map,
+                                                           const __grid_constant__ CUtensorMap q_map)
+{
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    __shared__ TcShared sh;
+    __shared__ int prefix[1025];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n_rb = p.rows_pad / 128, NS = p.tc_stages;
+    unsigned char *base = reinterpret_cast<unsigned char *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    unsigned char *Qs = base;                                   // [n_rb][2 halves][128 rows][128 B]
+    unsigned char *Ks = Qs + (size_t)n_rb * kTileBytes;         // [NS][2 halves][128 rows][128 B]
+    float *fin_s = reinterpret_cast<float *>(Ks + (size_t)NS * kTileBytes);   // [2][rows_pad]
+    float2 *red = reinterpret_cast<float2 *>(fin_s + 2 * p.rows_pad);         // [2][n_rb][128]
+    volatile int *abort_flag = &sh.abort_flag;
+
+    if (tid == 0) {
+        for (int i = 0; i < kMaxStages; ++i) { mbar_init(smem_u32(&sh.kfull[i]), 1); mbar_init(smem_u32(&sh.kempty[i]), 1); }
+        for (int i = 0; i < kSlots; ++i) { mbar_init(smem_u32(&sh.tfull[i]), 1); mbar_init(smem_u32(&sh.tempty[i]), 4); }
+        mbar_init(smem_u32(&sh.qfull), 1);
+        mbar_init(smem_u32(&sh.qempty), 1);
+        mbar_init(smem_u32(&sh.done), 1);
+        sh.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    tc_partition(p, gridDim.x, prefix, &sh.tiles_lh, &sh.n_tiles, &sh.tpc);
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)), "r"(512) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = sh.tmem_base;
+    const int tiles_lh = sh.tiles_lh, tpc = sh.tpc;
+    const long long g_begin = (long long)blockIdx.x * tpc;
+    const long long g_end = (g_begin + tpc < sh.n_tiles) ? g_begin + tpc : sh.n_tiles;
+    if (PHASE == 1 && blockIdx.x == 0 && tid == 0) {
+        for (int b = 0; b < p.B; ++b) {
+            const int T = p.seq_lens[b];
+            if (T > p.Tk && T <= p.T_cap && p.W > T) set_status(p.status, AMS_ERR_INVALID_ARG, b, p.W, T);
+        }
+    }
+    const float c = kLog2e * 0.08838834764831845f; // log2(e) / sqrt(128)
+
+    if (tiles_lh > 0 && g_begin < g_end) {
+        if (warp == 0) {
+            // ------------------------------------------------------------ TMA producer
+            int kit = 0, seg = 0, issued = 0;
+            bool ok = true;
+            for (long long g = g_begin; g < g_end && ok;) {
+                const Segment s = decode_segment(p, prefix, tiles_lh, tpc, g, g_end);
+                ok = mbar_wait(smem_u32(&sh.qempty), (uint32_t)((seg & 1) ^ 1), abort_flag);
+                if (!ok) break;
+                if (lane == 0) {
+                    mbar_expect_tx(smem_u32(&sh.qfull), (uint32_t)(n_rb * kTileBytes));
+                    const int qrow0 = ((s.l * p.B + s.b) * p.H * p.G + s.h * p.G) * p.W;
+                    for (int rb = 0; rb < n_rb; ++rb)
+                        for (int hf = 0; hf < 2; ++hf)
+                            tma_load_2d(smem_u32(Qs + (size_t)rb * kTileBytes + hf * kHalfBytes), &q_map, smem_u32(&sh.qfull),
+                                        hf * 64, qrow0 + rb * 128);
+                }
+                const int *table = p.block_table + (size_t)s.b * p.bt_stride;
+                const int last_page = (s.T - 1) >> 4;
+                for (int i = 0; i < s.n && ok; ++i, ++kit) {
+                    const int st = kit % NS;
+                    ok = mbar_wait(smem_u32(&sh.kempty[st]), (uint32_t)(((kit / NS) & 1) ^ 1), abort_flag);
+                    if (!ok) break;
+                    if (lane == 0) mbar_expect_tx(smem_u32(&sh.kfull[st]), (uint32_t)kTileBytes);
+                    __syncwarp();
+                    if (lane < 16) {
+                        const int pg = lane >> 1, hf = lane & 1;
+                        int pi = (s.tile0 + i) * 8 + pg;
+                        if (pi > last_page) pi = last_page;  // tokens past the end are masked by position
+                        tma_load_5d(smem_u32(Ks + (size_t)st * kTileBytes + hf * kHalfBytes + pg * 2048), &k_map,
+                                    smem_u32(&sh.kfull[st]), hf * 64, s.h, 0, table[pi], s.l);
+                    }
+                    issued = kit + 1;
+                }
+                g += s.n;
+                ++seg;
+            }
+            if (!ok) { // drain: wait (bounded) for the copies that were issued and never consumed
+                for (int k = max(0, issued - NS); k < issued; ++k) {
+                    for (uint32_t i = 0; i < kWaitLimit; ++i)
+                        if (mbar_try_wait(smem_u32(&sh.kfull[k % NS]), (uint32_t)((k / NS) & 1))) break;
+                }
+            }
+        } else if (warp == 1) {
+            // ------------------------------------------------------------ MMA issuer
+            if (lane == 0) {
+                int kit = 0, sit = 0, seg = 0;
+                bool ok = true;
+                for (long long g = g_begin; g < g_end && ok;) {
+                    const Segment s = decode_segment(p, prefix, tiles_lh, tpc, g, g_end);
+                    ok = mbar_wait(smem_u32(&sh.qfull), (uint32_t)(seg & 1), abort_flag);
+                    for (int i = 0; i < s.n && ok; ++i, ++kit) {
+                        const int st = kit % NS;
+                        ok = mbar_wait(smem_u32(&sh.kfull[st]), (uint32_t)((kit / NS) & 1), abort_flag);
+                        for (int rb = 0; rb < n_rb && ok; ++rb, ++sit) {
+                            const int slot = sit % kSlots;
+                            ok = mbar_wait(smem_u32(&sh.tempty[slot]), (uint32_t)(((sit / kSlots) & 1) ^ 1), abort_flag);
+                            if (!ok) break;
+                            tc_fence_after();
+                            const uint32_t qa = smem_u32(Qs + (size_t)rb * kTileBytes), ka = smem_u32(Ks + (size_t)st * kTileBytes);
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                const uint32_t off = (uint32_t)((k >> 2) * kHalfBytes + (k & 3) * 32);
+                                const unsigned long long dq = smem_desc(qa + off), dk = smem_desc(ka + off);
+                                tc_mma(tmem_base + (uint32_t)(slot * 128), PHASE == 1 ? dq : dk, PHASE == 1 ? dk : dq, kIdesc, k > 0);
+                            }
+                            tc_commit(smem_u32(&sh.tfull[slot]));
+                        }
+                        if (ok) tc_commit(smem_u32(&sh.kempty[st]));
+                    }
+                    if (ok) tc_commit(smem_u32(&sh.qempty));
+                    g += s.n;
+                    ++seg;
+                }
+                // all tensor work issued by this thread has finished before TMEM is released
+                tc_commit(smem_u32(&sh.done));
+                for (uint32_t i = 0; i < kWaitLimit; ++i)
+                    if (mbar_try_wait(smem_u32(&sh.done), 0)) break;
+            }
+            __syncwarp();
+        } else if (warp >= 4) {
+            // ------------------------------------------------------------ consumers
+            const int wg = (warp - 4) >> 2, quad = warp & 3, li = quad * 32 + lane; // li = TMEM lane of this thread
+            int kit = 0, sit = 0, seg = 0;
+            bool ok = true;
+            // a thread whose wait ran out keeps walking the segments without touching the pipeline, so that
+            // the consumers' named barriers stay matched
+            for (long long g = g_begin; g < g_end;) {
+                const Segment s = decode_segment(p, prefix, tiles_lh, tpc, g, g_end);
+                const int T = s.T;
+                float m[4], z[4];
+                int lastv[4];
+                const float *fin = p.fin + (size_t)s.uid * (p.rows_pad + 8);
+                float *fs = fin_s + (seg & 1) * p.rows_pad;
+                float pmax = 0.0f;
+                if (PHASE == 1) {
+#pragma unroll
+                    for (int rb = 0; rb < 4; ++rb) {
+                        m[rb] = -INFINITY; z[rb] = 0.0f;
+                        const int r = rb * 128 + li;
+                        lastv[rb] = r < p.rows ? (p.causal ? T - p.W + (r % p.W) : T - 1) : -1;
+                    }
+                } else {
+                    for (int r = (warp - 4) * 32 + lane; r < p.rows_pad; r += 256) fs[r] = fin[r];
+                    pmax = fin[p.rows_pad];
+                    asm volatile("bar.sync 1, 256;" ::: "memory");
+                }
+                for (int i = 0; i < s.n && ok; ++i, ++kit) {
+                    if ((kit & 1) != wg) { sit += n_rb; continue; }
+                    const int t0 = (s.tile0 + i) * kTileTokens;
+                    float acc = 0.0f;
+                    for (int rb = 0; rb < n_rb && ok; ++rb, ++sit) {
+                        const int slot = sit % kSlots;
+                        ok = mbar_wait(smem_u32(&sh.tfull[slot]), (uint32_t)((sit / kSlots) & 1), abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * 128);
+                        if (PHASE == 1) {
+                            const int lv = min(lastv[rb], T - 1);
+                            float mr = m[rb], zr = z[rb];
+#pragma unroll 1
+                            for (int ch = 0; ch < 4; ++ch) {
+                                float v[32];
+                                tc_ld32(taddr + ch * 32, v);
+                                const int tc0 = t0 + ch * 32;
+                                if (tc0 > lv) continue;
+                                if (tc0 + 31 > lv) {
+#pragma unroll
+                                    for (int j = 0; j < 32; ++j) if (tc0 + j > lv) v[j] = -INFINITY;
+                                }
+                                float cm = v[0];
+#pragma unroll
+                                for (int j = 1; j < 32; ++j) cm = fmaxf(cm, v[j]);
+                                const float mn = fmaxf(mr, cm * c);
+                                zr *= ex2(mr - mn);
+                                mr = mn;
+                                float zs = 0.0f;
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) zs += ex2(fmaf(v[j], c, -mn));
+                                zr += zs;
+                            }
+                            m[rb] = mr; z[rb] = zr;
+                        } else {
+                            const int t = t0 + li;
+                            const bool plain = !p.causal || t0 + kTileTokens - 1 <= T - p.W;
+                            const float *fr = fs + rb * 128;
+#pragma unroll 1
+                            for (int ch = 0; ch < 4; ++ch) {
+                                float v[32];
+                                tc_ld32(taddr + ch * 32, v);
+                                if (plain) {
+#pragma unroll
+                                    for (int j = 0; j < 32; ++j) acc += ex2(fmaf(v[j], c, -fr[ch * 32 + j]));
+                                } else {
+                                    const int rbase = rb * 128 + ch * 32;
+#pragma unroll
+                                    for (int j = 0; j < 32; ++j) {
+                                        const int r = rbase + j;
+                                        const bool seen = t <= T - p.W + (r % p.W);
+                                        acc += seen ? ex2(fmaf(v[j], c, -fr[ch * 32 + j])) : 0.0f;
+                                    }
+                                }
+                            }
+                        }
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&sh.tempty[slot]));
+                    }
+                    if (PHASE == 2 && ok) {
+                        const int t = t0 + li;
+                        if (t < T) {
+                            const int ninv = p.causal ? p.G * max(0, t - (T - p.W)) : 0;
+                            p.scores[(size_t)s.uid * p.T_cap + t] = (acc + (float)ninv * pmax) * (1.0f / (float)p.rows);
+                        }
+                    }
+                }
+                if (PHASE == 1) {
+                    // fold the two warpgroups' statistics and store this block's part of the unit
+                    float2 *rd = red + (size_t)(seg & 1) * n_rb * 128;
+                    if (wg == 1)
+                        for (int rb = 0; rb < n_rb; ++rb) rd[rb * 128 + li] = make_float2(m[rb], z[rb]);
+                    asm volatile("bar.sync 1, 256;" ::: "memory");
+                    if (wg == 0 && ok) {
+                        float2 *out = reinterpret_cast<float2 *>(p.part) + ((size_t)s.uid * p.n_slices + s.part) * p.rows_pad;
+                        for (int rb = 0; rb < n_rb; ++rb) {
+                            const float2 o = rd[rb * 128 + li];
+                            float mm = m[rb], zz = z[rb];
+                            lse_merge(mm, zz, o.x, o.y);
+                            out[rb * 128 + li] = make_float2(mm, zz);
+                        }
+                    }
+                }
+                g += s.n;
+                ++seg;
+            }
+        }
+    }
+    if (*abort_flag && tid == 0) set_status(p.status, AMS_ERR_TIMEOUT, blockIdx.x, PHASE, 0);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+}
+
+// Per unit: merge the parts written by the blocks that shared the unit, in block order.
+__global__ void __launch_bounds__(128) k_tova_combine_tc(DevParams p, int tc_grid)
+{
+    __shared__ u64 scratch[40];
+    __shared__ int prefix[1025];
+    __shared__ int s_tiles_lh, s_tpc;
+    __shared__ long long s_n;
+    tc_partition(p, tc_grid, prefix, &s_tiles_lh, &s_n, &s_tpc);
+    const int uid = blockIdx.x;
+    const int h = uid % p.H, b = (uid / p.H) % p.B, l = uid / (p.H * p.B);
+    const int nt = prefix[b + 1] - prefix[b];
+    if (nt == 0) return;
+    const long long ustart = (long long)(l * p.H + h) * s_tiles_lh + prefix[b];
+    const int n_parts = (int)((ustart + nt - 1) / s_tpc) - (int)(ustart / s_tpc) + 1;
+    float *fin = p.fin + (size_t)uid * (p.rows_pad + 8);
+    float best = 0.0f;
+    for (int r = threadIdx.x; r < p.rows_pad; r += blockDim.x) {
+        float m = -INFINITY, z = 0.0f;
+        for (int s = 0; s < n_parts; ++s) {
+            const float2 v = reinterpret_cast<const float2 *>(p.part)[((size_t)uid * p.n_slices + s) * p.rows_pad + r];
+            lse_merge(m, z, v.x, v.y);
+        }
+        if (r < p.rows && z > 0.0f) {
+            fin[r] = m + log2f(z);
+            best = fmaxf(best, 1.0f / z);
+        } else {
+            fin[r] = INFINITY;
+        }
+    }
+    best = block_max_f32(best, scratch);
+    if (threadIdx.x == 0) fin[p.rows_pad] = best;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)ptr;
+    }
+    return fn;
+}
+
+} // namespace
+
+bool tova_tc_supported(const DevParams &p) { return p.rows >= 64 && p.rows_pad % 128 == 0 && p.rows_pad <= 512 && p.B <= 1024; }
+
+size_t tova_tc_smem_bytes(const DevParams &p)
+{
+    return 1024 + (size_t)(p.rows_pad / 128 + p.tc_stages) * kTileBytes + (size_t)2 * p.rows_pad * 4 +
+           (size_t)2 * (p.rows_pad / 128) * 128 * 8 + 256;
+}
+
+int launch_score_tova_tc(const DevParams &p, LaunchCtx &ctx)
+{
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return AMS_ERR_CUDA;
+    CUtensorMap k_map, q_map;
+    {
+        const cuuint64_t dims[5] = {kHeadDim, (cuuint64_t)p.H, kPage, (cuuint64_t)p.num_pages, (cuuint64_t)p.L};
+        const cuuint64_t strides[4] = {kRowBytes, (cuuint64_t)p.H * kRowBytes, (cuuint64_t)kPage * p.H * kRowBytes,
+                                       (cuuint64_t)p.num_pages * kPage * p.H * kRowBytes};
+        const cuuint32_t box[5] = {64, 1, kPage, 1, 1};
+        const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+        if (enc(&k_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, p.k_pages, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return AMS_ERR_CUDA;
+    }
+    {
+        const cuuint64_t dims[2] = {kHeadDim, (cuuint64_t)p.L * p.B * p.H * p.G * p.W};
+        const cuuint64_t strides[1] = {kRowBytes};
+        const cuuint32_t box[2] = {64, 128};
+        const cuuint32_t estr[2] = {1, 1};
+        if (enc(&q_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16 *>(p.q), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return AMS_ERR_CUDA;
+    }
+    static int n_sm = 0;
+    if (!n_sm) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return AMS_ERR_CUDA;
+    }
+    const size_t smem = tova_tc_smem_bytes(p);
+    static size_t configured = 0;
+    if (smem > configured) {
+        if (cudaFuncSetAttribute(k_tova_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+            cudaFuncSetAttribute(k_tova_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return AMS_ERR_CUDA;
+        configured = smem;
+    }
+    const long long cap_tiles = (long long)p.L * p.B * p.H * ((p.T_cap + kTileTokens - 1) / kTileTokens);
+    long long want = (cap_tiles + p.tc_tpc_min - 1) / p.tc_tpc_min;
+    const int grid = (int)(want < n_sm ? (want < 1 ? 1 : want) : n_sm);
+    k_tova_tc<1><<<grid, kTcThreads, smem, ctx.s>>>(p, k_map, q_map);
+    ctx.mark(kKernScore1);
+    k_tova_combine_tc<<<p.L * p.B * p.H, 128, 0, ctx.s>>>(p, grid);
+    ctx.mark(kKernScoreCombine);
+    k_tova_tc<2><<<grid, kTcThreads, smem, ctx.s>>>(p, k_map, q_map);
+    ctx.mark(kKernScore2);
+    return cudaGetLastError() == cudaSuccess ? AMS_OK : AMS_ERR_CUDA;
+}
+
+} // namespace ams

@@ -146,6 +146,9 @@ def _check_scorer(wl, rtol=1e-3, atol=0.0, sample_units=None):
     (5, (32, 8), 1500, "rows20_window"),
     (32, (32, 8), 2100, "rows128_window"),
     (24, (64, 8), 1333, "rows192_two_row_blocks"),
+    (16, (32, 8), 1100, "rows64_padded_to_128"),
+    (64, (64, 8), 2309, "rows512_four_row_blocks"),
+    (32, (32, 8), 5000, "rows128_window_long"),
 ])
 def test_tova_scores_and_selection(window, group_heads, T, name):
     wl = _small(0, n_layers=1, batch=2, seq_len_min=T, seq_len_max=T, window=window, n_q_heads=group_heads[0],
