@@ -6,7 +6,8 @@
 //   warp 0      TMA producer: query block of the current unit, then one 32 KB K tile per
 //               stage (eight 16-token pages, two 64-wide halves each, 128-byte swizzle);
 //   warp 1      MMA issuer (one lane): per (tile, 128-row query block) eight
-//               tcgen05.mma m128 n128 k16 into one of four 128-column TMEM slots;
+//               tcgen05.mma m128 n128 k16 into one of four 128-column TMEM slots (two per
+//               consumer warpgroup, used in turn);
 //   warps 4-11  two consumer warpgroups, alternating tiles; thread i of a warpgroup owns
 //               TMEM lane i of its slots.
 // Phase 1 puts query rows on the TMEM lanes (A = Q, B = K), so a thread folds its row's
@@ -270,7 +271,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
         } else if (warp == 1) {
             // ------------------------------------------------------------ MMA issuer
             if (lane == 0) {
-                int kit = 0, sit = 0, seg = 0;
+                int kit = 0, seg = 0;
+                int wsit[2] = {0, 0}; // accumulator slots handed to each consumer warpgroup so far
                 bool ok = true;
                 for (long long g = g_begin; g < g_end && ok;) {
                     const Segment s = decode_segment(p, prefix, tiles_lh, tpc, g, g_end);
@@ -278,9 +280,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
                     for (int i = 0; i < s.n && ok; ++i, ++kit) {
                         const int st = kit % NS;
                         ok = mbar_wait(smem_u32(&sh.kfull[st]), (uint32_t)((kit / NS) & 1), abort_flag);
-                        for (int rb = 0; rb < n_rb && ok; ++rb, ++sit) {
-                            const int slot = sit % kSlots;
-                            ok = mbar_wait(smem_u32(&sh.tempty[slot]), (uint32_t)(((sit / kSlots) & 1) ^ 1), abort_flag);
+                        const int wg = kit & 1;
+                        for (int rb = 0; rb < n_rb && ok; ++rb, ++wsit[wg]) {
+                            // warpgroup wg owns slots 2 wg and 2 wg + 1, used in turn
+                            const int slot = 2 * wg + (wsit[wg] & 1);
+                            ok = mbar_wait(smem_u32(&sh.tempty[slot]), (uint32_t)(((wsit[wg] >> 1) & 1) ^ 1), abort_flag);
                             if (!ok) break;
                             tc_fence_after();
                             const uint32_t qa = smem_u32(Qs + (size_t)rb * kTileBytes), ka = smem_u32(Ks + (size_t)st * kTileBytes);
@@ -307,7 +311,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
         } else if (warp >= 4) {
             // ------------------------------------------------------------ consumers
             const int wg = (warp - 4) >> 2, quad = warp & 3, li = quad * 32 + lane; // li = TMEM lane of this thread
-            int kit = 0, sit = 0, seg = 0;
+            int kit = 0, wsit = 0, seg = 0;
             bool ok = true;
             // a thread whose wait ran out keeps walking the segments without touching the pipeline, so that
             // the consumers' named barriers stay matched
@@ -332,12 +336,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
                     asm volatile("bar.sync 1, 256;" ::: "memory");
                 }
                 for (int i = 0; i < s.n && ok; ++i, ++kit) {
-                    if ((kit & 1) != wg) { sit += n_rb; continue; }
+                    if ((kit & 1) != wg) continue;
                     const int t0 = (s.tile0 + i) * kTileTokens;
                     float acc = 0.0f;
-                    for (int rb = 0; rb < n_rb && ok; ++rb, ++sit) {
-                        const int slot = sit % kSlots;
-                        ok = mbar_wait(smem_u32(&sh.tfull[slot]), (uint32_t)((sit / kSlots) & 1), abort_flag);
+                    for (int rb = 0; rb < n_rb && ok; ++rb, ++wsit) {
+                        const int slot = 2 * wg + (wsit & 1);
+                        ok = mbar_wait(smem_u32(&sh.tfull[slot]), (uint32_t)((wsit >> 1) & 1), abort_flag);
                         if (!ok) break;
                         tc_fence_after();
                         const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * 128);
