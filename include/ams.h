@@ -123,7 +123,7 @@ int ams_init_state(const ams_config *cfg, void *ema_state, void *workspace, size
  *  obs_queries, window : may be NULL / 0 for AMS_SCORER_KEYDIFF and AMS_SCORER_EXTERNAL.
  *  ema_state        : the buffer given to ams_init_state (or a restored copy of it).
  *  n_segments       : S, the number of mass quantiles (segment mass 1/S), 1..max_segments.
- *  ext_scores       : AMS_SCORER_EXTERNAL only: fp32 [L][batch][H][max_seq_len] scores used both
+ *  ext_scores       : AMS_SCORER_EXTERNAL only: fp32 [L][batch][H][max_seq_len] (16-byte aligned) scores used both
  *                     as usage and as base scores.
  *  dbg              : optional views, or NULL.
  * Calls on the same handle share the workspace and must not overlap on the GPU. */

@@ -196,7 +196,7 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
     } else if (scorer_id != AMS_SCORER_KEYDIFF) {
         return AMS_ERR_INVALID_ARG;
     }
-    if (((uintptr_t)k_pages | (uintptr_t)v_pages | (uintptr_t)obs_queries | (uintptr_t)ema_state) & 15) return AMS_ERR_INVALID_ARG;
+    if (((uintptr_t)k_pages | (uintptr_t)v_pages | (uintptr_t)obs_queries | (uintptr_t)ema_state | (uintptr_t)ext_scores) & 15) return AMS_ERR_INVALID_ARG;
 
     const Layout &y = st->lay;
     cudaStream_t s = (cudaStream_t)stream;
@@ -234,7 +234,7 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
     ctx.begin();
     if (scorer_id == AMS_SCORER_TOVA) rc = launch_score_tova(p, ctx);
     else if (scorer_id == AMS_SCORER_KEYDIFF) rc = launch_score_keydiff(p, ctx);
-    if (rc == AMS_OK) rc = launch_segment_select(p, ctx);
+    if (rc == AMS_OK) rc = segment_cluster_supported(p) ? launch_segment_select_cluster(p, ctx) : launch_segment_select(p, ctx);
     if (rc == AMS_OK && dbg) {
         // inspection copies are taken before the table is rewritten
         const size_t U = (size_t)p.L * p.B * p.H;

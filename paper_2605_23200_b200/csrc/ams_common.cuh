@@ -196,6 +196,8 @@ size_t tova_tc_smem_bytes(const DevParams &p);
 int launch_score_tova_tc(const DevParams &p, LaunchCtx &ctx);
 int launch_score_keydiff(const DevParams &p, LaunchCtx &ctx);
 int launch_segment_select(const DevParams &p, LaunchCtx &ctx);
+bool segment_cluster_supported(const DevParams &p);
+int launch_segment_select_cluster(const DevParams &p, LaunchCtx &ctx);
 int launch_gather(const DevParams &p, LaunchCtx &ctx);
 
 } // namespace ams

@@ -1,0 +1,667 @@
+// Algorithm 1 steps 1-5 of the paper (mass, EMA credit, prefix scan, cuts, merge/split,
+// quotas, per-segment top-q, must-keep, backfill, ordered index compaction) with every
+// per-token array held on chip.
+//
+// One thread-block cluster handles one (layer, sequence, KV head).  Block r of the cluster
+// owns tokens [r * TPC, (r + 1) * TPC); thread i of a block owns VPT consecutive tokens,
+// whose fixed-point masses, sort keys and credits live in registers / thread-private shared
+// memory.  Every per-token step is done by the owning thread on this block's shared memory;
+// the blocks of a cluster meet only to add up per-block sums and per-segment counts through
+// distributed shared memory.  Results are bit-identical to the one-block kernel: all
+// decisions are integer, and integer sums do not depend on their order.
+#include <cooperative_groups.h>
+#include <string.h>
+
+#include "ams_common.cuh"
+#include "ams_select.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace ams {
+
+using namespace sel;
+
+namespace {
+
+constexpr int kXch = 8; // ring of exchange slots (>= 2)
+
+// Dynamic shared memory of one block (byte offsets).
+struct SmemMap {
+    size_t gs, flags, crs, cend, ms, bounds, quota, cap, give, raw, merged, poff, cand, cnt, take, ties, tps, qthr, total;
+};
+
+__host__ __device__ inline size_t up16(size_t x) { return (x + 15) & ~(size_t)15; }
+
+__host__ __device__ inline SmemMap smem_map(int tpc, int sc, int S, bool ema_on)
+{
+    SmemMap m;
+    size_t o = 0;
+    m.gs = o;     o = up16(o + (size_t)tpc * 4);
+    m.flags = o;  o = up16(o + (size_t)tpc);
+    m.crs = o;    o = up16(o + (ema_on ? (size_t)tpc * 4 : 0));
+    m.cend = o;   o = up16(o + (size_t)(sc + 1) * 8);
+    m.ms = o;     o = up16(o + (size_t)sc * 8);
+    m.bounds = o; o = up16(o + (size_t)(sc + 1) * 4);
+    m.quota = o;  o = up16(o + (size_t)sc * 4);
+    m.cap = o;    o = up16(o + (size_t)sc * 4);
+    m.give = o;   o = up16(o + (size_t)sc * 4);
+    m.raw = o;    o = up16(o + (size_t)(S + 1) * 4);
+    m.merged = o; o = up16(o + (size_t)(S + 1) * 4);
+    m.poff = o;   o = up16(o + (size_t)(S + 1) * 4);
+    m.cand = o;   o = up16(o + (size_t)sc * 4);
+    m.cnt = o;    o = up16(o + (size_t)2 * 3 * sc * 4);
+    m.take = o;   o = up16(o + (size_t)sc * 4);
+    m.ties = o;   o = up16(o + (size_t)sc * 4);
+    m.tps = o;    o = up16(o + (size_t)sc * 4);
+    m.qthr = o;   o = up16(o + (size_t)(S + 1) * 8);
+    m.total = o;
+    return m;
+}
+
+template <int NT, int VPT>
+__global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, int cs)
+{
+    constexpr int nt = NT, TPC = NT * VPT;
+    extern __shared__ __align__(16) unsigned char dyn[];
+    __shared__ Smem sm;
+    __shared__ u64 xch[kXch];
+    cg::cluster_group cluster = cg::this_cluster();
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int rank = cs > 1 ? (int)cluster.block_rank() : 0;
+    const int uid = blockIdx.x / cs;
+    const int h = uid % p.H, b = (uid / p.H) % p.B, l = uid / (p.H * p.B);
+    const int T = p.seq_lens[b];
+    // every exit below is taken by all blocks of the cluster together
+    if (T <= p.Tk) return; // nothing to evict
+    if (T > p.T_cap) { if (tid == 0 && rank == 0) set_status(p.status, AMS_ERR_CAPACITY, uid, T, p.T_cap); return; }
+
+    const int sc = p.seg_cap;
+    const bool ema_on = p.beta != 1.0f;
+    const SmemMap mp = smem_map(TPC, sc, p.S, ema_on);
+    float *gs = reinterpret_cast<float *>(dyn + mp.gs);
+    unsigned char *flags = dyn + mp.flags;
+    float *crs = reinterpret_cast<float *>(dyn + mp.crs);      // [VPT][nt], thread-private columns
+    u64 *Cend = reinterpret_cast<u64 *>(dyn + mp.cend);
+    u64 *Ms = reinterpret_cast<u64 *>(dyn + mp.ms);
+    int *bounds = reinterpret_cast<int *>(dyn + mp.bounds);
+    int *quota = reinterpret_cast<int *>(dyn + mp.quota);
+    int *cap = reinterpret_cast<int *>(dyn + mp.cap);
+    int *give = reinterpret_cast<int *>(dyn + mp.give);
+    int *raw = reinterpret_cast<int *>(dyn + mp.raw);
+    int *merged = reinterpret_cast<int *>(dyn + mp.merged);
+    int *poff = reinterpret_cast<int *>(dyn + mp.poff);
+    unsigned *cand = reinterpret_cast<unsigned *>(dyn + mp.cand);
+    int *cnt = reinterpret_cast<int *>(dyn + mp.cnt);
+    int *takev = reinterpret_cast<int *>(dyn + mp.take);
+    int *tiesv = reinterpret_cast<int *>(dyn + mp.ties);
+    int *tps = reinterpret_cast<int *>(dyn + mp.tps);
+    u64 *qthr = reinterpret_cast<u64 *>(dyn + mp.qthr);
+
+    const int t_base = rank * TPC;                       // first token of this block
+    const int n_loc = max(0, min(TPC, T - t_base));      // tokens of this block
+    const int my0 = tid * VPT;                           // local index of this thread's first token
+    const size_t row = (size_t)uid * p.T_cap;
+    float *credit = p.ema + (((size_t)l * p.Bmax + b) * p.H + h) * (size_t)p.T_cap;
+    int *keep = p.keep_idx + (size_t)uid * p.Tk;
+    const double two_f = (double)(1ull << kFixBits);
+    int xn = 0; // exchanges done so far (same in every thread of the cluster)
+
+    auto unit_barrier = [&]() { if (cs > 1) cluster.sync(); else __syncthreads(); };
+    // Sum over the whole sequence; *prefix (optional) = sum over the blocks before this one.
+    // A slot of the ring is rewritten only after kXch - 1 later cluster barriers, which every
+    // block reaches only after it has read the slot.
+    auto unit_sum = [&](u64 v, u64 *prefix) -> u64 {
+        const u64 mine = block_sum_u64(v, sm.scratch);
+        if (prefix) *prefix = 0;
+        if (cs == 1) return mine;
+        u64 *slot = &xch[xn++ % kXch];
+        if (tid == 0) *slot = mine;
+        cluster.sync();
+        u64 tot = 0;
+        for (int r = 0; r < cs; ++r) {
+            const u64 x = *cluster.map_shared_rank(slot, r);
+            if (prefix && r < rank) *prefix += x;
+            tot += x;
+        }
+        return tot;
+    };
+    auto unit_max = [&](float v) -> float {
+        const float mine = block_max_f32(v, sm.scratch);
+        if (cs == 1) return mine;
+        u64 *slot = &xch[xn++ % kXch];
+        if (tid == 0) *slot = (u64)__float_as_uint(mine);
+        cluster.sync();
+        float m = mine;
+        for (int r = 0; r < cs; ++r) m = fmaxf(m, __uint_as_float((unsigned)*cluster.map_shared_rank(slot, r)));
+        return m;
+    };
+
+    // ---- scores into shared memory (token order); cut table starts at "no cut"
+    {
+        const float *g = p.scores + row + t_base;
+        for (int i = tid * 4; i < n_loc; i += nt * 4)
+            *reinterpret_cast<float4 *>(gs + i) = *reinterpret_cast<const float4 *>(g + i);
+        for (int k = tid; k <= p.S; k += nt) raw[k] = T;
+    }
+    __syncthreads();
+
+    // ---- Eq. 1 weights of this thread's tokens (re-read from shared memory where needed,
+    //      so that they do not occupy registers across the reductions)
+    auto load_w = [&](float (&w)[VPT]) {
+#pragma unroll
+        for (int q = 0; q < VPT / 4; ++q) {
+            float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            if (my0 + 4 * q < n_loc) v = *reinterpret_cast<const float4 *>(gs + my0 + 4 * q);
+            w[4 * q] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
+        }
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) w[i] = (my0 + i < n_loc) ? weight_of(w[i], p.eps) : 0.0f;
+    };
+    if (ema_on) {
+#pragma unroll
+        for (int q = 0; q < VPT / 4; ++q) {
+            float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            if (my0 + 4 * q < n_loc) v = *reinterpret_cast<const float4 *>(credit + t_base + my0 + 4 * q);
+            crs[(4 * q) * nt + tid] = v.x; crs[(4 * q + 1) * nt + tid] = v.y;
+            crs[(4 * q + 2) * nt + tid] = v.z; crs[(4 * q + 3) * nt + tid] = v.w;
+        }
+    }
+    float wmax = 0.0f;
+    {
+        float w[VPT];
+        load_w(w);
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) wmax = fmaxf(wmax, w[i]);
+    }
+    wmax = unit_max(wmax);
+    const double sw = fix_scale(wmax);
+    u64 sa = 0;
+    {
+        float w[VPT];
+        load_w(w);
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) sa += to_fixed(w[i], sw);
+    }
+    const u64 SA = unit_sum(sa, nullptr);
+    const double dSA = (double)SA;
+
+    // ---- EMA credit and the fixed-point mass used for segmentation
+    float *mass_dbg = p.mass_dbg ? p.mass_dbg + row + t_base + my0 : nullptr;
+    u64 Hm[VPT];
+    if (ema_on) {
+        const float oml = __fsub_rn(1.0f, p.lambda);
+        float cmax = 0.0f;
+        float w[VPT];
+        load_w(w);
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            if (my0 + i < n_loc) {
+                const u64 A = to_fixed(w[i], sw);
+                const float m = __double2float_rn(__ddiv_rn((double)A, dSA));
+                const float cn = __fadd_rn(__fmul_rn(p.lambda, crs[i * nt + tid]), __fmul_rn(oml, m));
+                crs[i * nt + tid] = cn;
+                if (mass_dbg) mass_dbg[i] = m;
+                cmax = fmaxf(cmax, cn);
+            }
+        }
+        cmax = unit_max(cmax);
+        u64 scsum = 0;
+        double scl = 0.0;
+        if (cmax > 0.0f) {
+            scl = fix_scale(cmax);
+#pragma unroll
+            for (int i = 0; i < VPT; ++i)
+                if (my0 + i < n_loc) scsum += to_fixed(crs[i * nt + tid], scl);
+        }
+        const u64 SC = unit_sum(scsum, nullptr);
+        const double dSC = (double)SC, bd = (double)p.beta, omb = __dsub_rn(1.0, (double)p.beta);
+        load_w(w);
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            Hm[i] = 0;
+            if (my0 + i < n_loc) {
+                const u64 A = to_fixed(w[i], sw);
+                const double cur = __dmul_rn(bd, __ddiv_rn((double)A, dSA));
+                double hist_term = 0.0;
+                if (SC > 0) hist_term = __dmul_rn(omb, __ddiv_rn((double)to_fixed(crs[i * nt + tid], scl), dSC));
+                Hm[i] = (u64)__double2ull_rd(__dmul_rn(__dadd_rn(cur, hist_term), two_f));
+            }
+        }
+    } else {
+        float w[VPT];
+        load_w(w);
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            Hm[i] = 0;
+            if (my0 + i < n_loc) {
+                const u64 A = to_fixed(w[i], sw);
+                const double r = __ddiv_rn((double)A, dSA);
+                if (mass_dbg) mass_dbg[i] = __double2float_rn(r);
+                Hm[i] = (u64)__double2ull_rd(__dmul_rn(r, two_f));
+            }
+        }
+    }
+    u64 tt = 0;
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) tt += Hm[i];
+    u64 rank_prefix;
+    const u64 SH = unit_sum(tt, &rank_prefix);
+
+    // ---- prefix sum and mass-quantile cuts: the token that reaches quantile k closes its
+    //      segment, so the boundary is (position + 1); every block receives every cut.
+    //      C reaches quantile k when C * S >= k * SH, i.e. C >= ceil(k * SH / S)
+    const u64 S = (u64)p.S;
+    for (int k = tid + 1; k < p.S; k += nt) qthr[k] = ((u64)k * SH + S - 1) / S;
+    u64 btot;
+    const u64 exc = rank_prefix + block_excl_scan_u64(tt, sm.scratch, &btot); // (synchronises the block)
+    auto quantile = [&](u64 C) -> int { // number of k in [1, S) with qthr[k] <= C
+        int lo = 0, hi = p.S - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (qthr[mid] <= C) lo = mid; else hi = mid - 1;
+        }
+        return lo;
+    };
+    if (my0 < n_loc) {
+        int kprev = quantile(exc);
+        const int klast = quantile(exc + tt);
+        if (klast != kprev) {
+            u64 run = exc;
+#pragma unroll
+            for (int i = 0; i < VPT; ++i) {
+                if (my0 + i < n_loc) {
+                    run += Hm[i];
+                    const int kc = quantile(run);
+                    for (int k = kprev + 1; k <= kc; ++k) {
+                        const int cut = t_base + my0 + i + 1;
+                        if (cs == 1) raw[k] = cut;
+                        else for (int r = 0; r < cs; ++r) *cluster.map_shared_rank(raw + k, r) = cut;
+                    }
+                    kprev = kc;
+                }
+            }
+        }
+    }
+    unit_barrier();
+
+    // ---- merge short raw segments forward, fold a short tail left, count split pieces
+    //      (every block does this on its own copy of the cuts)
+    if (tid == 0) {
+        int nm = 0;
+        merged[nm++] = 0;
+        int last = 0;
+        for (int k = 1; k < p.S; ++k) {
+            const int e = raw[k];
+            if (e <= last || e >= T) continue;
+            last = e;
+            if (e - merged[nm - 1] >= p.l_min) merged[nm++] = e;
+        }
+        merged[nm++] = T;
+        if (nm > 2 && merged[nm - 1] - merged[nm - 2] < p.l_min) { merged[nm - 2] = T; --nm; }
+        int off = 0;
+        for (int i = 0; i + 1 < nm; ++i) {
+            const int len = merged[i + 1] - merged[i];
+            poff[i] = off;
+            off += (p.l_max > 0 && len > p.l_max) ? (len + p.l_max - 1) / p.l_max : 1;
+        }
+        poff[nm - 1] = off;
+        sm.bcast[0] = nm - 1;
+        sm.bcast[1] = off;
+    }
+    __syncthreads();
+    const int n_merged = sm.bcast[0], n_seg = sm.bcast[1];
+    if (n_seg > sc) { if (tid == 0 && rank == 0) set_status(p.status, AMS_ERR_CAPACITY, uid, n_seg, sc); return; }
+    if (tid == 0) bounds[0] = 0;
+    for (int i = 0; i < n_merged; ++i) {
+        const int a = merged[i], len = merged[i + 1] - a, pieces = poff[i + 1] - poff[i];
+        const int bs = len / pieces, extra = len % pieces;
+        for (int j = tid; j < pieces; j += nt) bounds[poff[i] + j + 1] = a + (j + 1) * bs + min(j + 1, extra);
+    }
+    __syncthreads();
+
+    // ---- segment of each of this thread's tokens: s0 = segment of the first one, bit i of
+    //      newseg = token i starts the next segment
+    unsigned valid = 0;
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) if (my0 + i < n_loc) valid |= 1u << i;
+    int seg0 = n_seg - 1;
+    unsigned newseg = 0;
+    if (valid) {
+        const int t0 = t_base + my0;
+        int lo = 0, hi = n_seg; // bounds[lo] <= t0 < bounds[hi]
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (bounds[mid] <= t0) lo = mid; else hi = mid;
+        }
+        seg0 = lo;
+        int s = lo, nb = bounds[lo + 1];
+#pragma unroll
+        for (int i = 1; i < VPT; ++i)
+            if (((valid >> i) & 1u) && t0 + i == nb) { newseg |= 1u << i; ++s; nb = bounds[s + 1]; }
+    }
+
+    // ---- prefix of the mass at each segment end, written by the thread that owns the
+    //      segment's last token; segment mass = difference of consecutive ends
+    if (valid) {
+        int s = seg0;
+        u64 run = exc;
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            if ((valid >> i) & 1u) {
+                if (i > 0 && ((newseg >> i) & 1u)) ++s;
+                run += Hm[i];
+                const bool ends = (i + 1 < VPT && ((newseg >> (i + 1)) & 1u)) || t_base + my0 + i + 1 == bounds[s + 1];
+                if (ends) {
+                    if (cs == 1) Cend[s] = run;
+                    else for (int r = 0; r < cs; ++r) *cluster.map_shared_rank(Cend + s, r) = run;
+                }
+            }
+        }
+    }
+    unit_barrier();
+
+    // ---- must-keep sizes and quotas (every block, same result)
+    const int ns = max(0, min(p.n_sink, min(p.Tk, T)));
+    const int nl = max(0, min(p.n_last, min(p.Tk - ns, T - ns)));
+    const int Bq = p.Tk - ns - nl;
+    long long smin = 0;
+    for (int i = tid; i < n_seg; i += nt) {
+        Ms[i] = Cend[i] - (i > 0 ? Cend[i - 1] : 0ull);
+        smin += max(0, min(p.q_min, bounds[i + 1] - bounds[i]));
+    }
+    smin = block_sum_i64(smin, sm.scratch);
+    const long long Trem = (long long)Bq - smin;
+    long long sq = 0;
+    for (int i = tid; i < n_seg; i += nt) {
+        const int L = bounds[i + 1] - bounds[i];
+        long long qi = max(0, min(p.q_min, L));
+        if (Trem >= 0) qi += (long long)((2ull * (u64)Trem * Ms[i] + SH) / (2ull * SH));
+        if (qi > L) qi = L;
+        quota[i] = (int)qi;
+        sq += qi;
+    }
+    sq = block_sum_i64(sq, sm.scratch);
+    const long long Dq = (long long)Bq - sq;
+    if (Dq > 0) {
+        for (int i = tid; i < n_seg; i += nt) cap[i] = bounds[i + 1] - bounds[i] - quota[i];
+        __syncthreads();
+        distribute<true>(Dq, cap, give, Ms, n_seg, sm);
+        for (int i = tid; i < n_seg; i += nt) quota[i] += give[i];
+    } else if (Dq < 0) {
+        for (int i = tid; i < n_seg; i += nt)
+            cap[i] = quota[i] - max(0, min(p.q_min, bounds[i + 1] - bounds[i]));
+        __syncthreads();
+        const long long left = distribute<false>(-Dq, cap, give, Ms, n_seg, sm);
+        for (int i = tid; i < n_seg; i += nt) quota[i] -= give[i];
+        if (left > 0) { // the budget cannot cover the minima: go below them
+            __syncthreads();
+            for (int i = tid; i < n_seg; i += nt) cap[i] = quota[i];
+            __syncthreads();
+            distribute<false>(left, cap, give, Ms, n_seg, sm);
+            for (int i = tid; i < n_seg; i += nt) quota[i] -= give[i];
+        }
+    }
+    __syncthreads();
+    if (rank == 0) {
+        if (tid == 0) p.n_seg[uid] = n_seg;
+        for (int i = tid; i < n_seg; i += nt) {
+            p.seg_bounds[(size_t)uid * (sc + 1) + i] = bounds[i];
+            p.quotas[(size_t)uid * sc + i] = quota[i];
+        }
+        if (tid == 0) p.seg_bounds[(size_t)uid * (sc + 1) + n_seg] = T;
+    }
+
+    // ---- selection machinery.
+    //      seg_search finds, for all segments at once, the q_s-th largest key of each segment
+    //      by fixing two key bits per round from the top: in a round every thread counts, per
+    //      segment it touches, its active tokens whose key is at least prefix | j << shift
+    //      (j = 1, 2, 3); one thread per segment then keeps the largest j that still leaves q_s
+    //      keys at or above.  A last round counts keys >= and > the final value, which gives
+    //      how many of the keys equal to it belong to the top q_s.  The count tables of even
+    //      and odd rounds alternate, so one cluster barrier per round is enough.
+    unsigned key[VPT];
+#pragma unroll
+    for (int q = 0; q < VPT / 4; ++q) {
+        float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        if (my0 + 4 * q < n_loc) v = *reinterpret_cast<const float4 *>(gs + my0 + 4 * q);
+        key[4 * q] = score_key(v.x); key[4 * q + 1] = score_key(v.y);
+        key[4 * q + 2] = score_key(v.z); key[4 * q + 3] = score_key(v.w);
+    }
+    auto seg_search = [&](const int *quo, int nsg, unsigned act, int s0, unsigned nsb) {
+        for (int s = tid; s < nsg; s += nt) cand[s] = 0u;
+        for (int i = tid; i < nsg * 3; i += nt) { cnt[i] = 0; cnt[sc * 3 + i] = 0; }
+        if (tid == 0) sm.bcast[7] = 0;
+        const bool wuni = __all_sync(0xffffffffu, nsb == 0 && s0 == __shfl_sync(0xffffffffu, s0, 0));
+        __syncthreads();
+        int par = 0;
+        for (int shift = 30; shift >= -2; shift -= 2, par ^= 1) {
+            const bool fin = shift < 0;
+            int *c = cnt + par * sc * 3;
+            int s = s0, c1 = 0, c2 = 0, c3 = 0;
+            auto flush = [&]() {
+                if (c1) atomicAdd(&c[s * 3], c1);
+                if (c2) atomicAdd(&c[s * 3 + 1], c2);
+                if (c3) atomicAdd(&c[s * 3 + 2], c3);
+            };
+            if (act) {
+                unsigned P = cand[s];
+#pragma unroll
+                for (int i = 0; i < VPT; ++i) {
+                    if (i > 0 && ((nsb >> i) & 1u)) {
+                        flush();
+                        ++s; c1 = c2 = c3 = 0;
+                        P = cand[s];
+                    }
+                    if ((act >> i) & 1u) {
+                        const unsigned k = key[i];
+                        if (!fin) {
+                            c1 += k >= (P | (1u << shift));
+                            c2 += k >= (P | (2u << shift));
+                            c3 += k >= (P | (3u << shift));
+                        } else {
+                            c1 += k >= P;
+                            c2 += k > P;
+                        }
+                    }
+                }
+            }
+            if (wuni) {
+                c1 = __reduce_add_sync(0xffffffffu, c1);
+                c2 = __reduce_add_sync(0xffffffffu, c2);
+                c3 = __reduce_add_sync(0xffffffffu, c3);
+                if (lane == 0) flush();
+            } else if (act) {
+                flush();
+            }
+            unit_barrier();
+            for (int sg = tid; sg < nsg; sg += nt) {
+                int a1 = c[sg * 3], a2 = c[sg * 3 + 1], a3 = c[sg * 3 + 2];
+                if (cs > 1) {
+                    a1 = a2 = a3 = 0;
+                    for (int r = 0; r < cs; ++r) {
+                        const int *rc = cluster.map_shared_rank(c + sg * 3, r);
+                        a1 += rc[0]; a2 += rc[1]; a3 += rc[2];
+                    }
+                }
+                const int q = quo[sg];
+                if (!fin) {
+                    const unsigned j = a3 >= q ? 3u : (a2 >= q ? 2u : (a1 >= q ? 1u : 0u));
+                    cand[sg] |= j << shift;
+                } else {
+                    takev[sg] = q - a2;       // keys equal to the threshold that belong to the top q
+                    tiesv[sg] = a1 - a2;      // keys equal to the threshold
+                    if (q - a2 < a1 - a2) sm.bcast[7] = 1;
+                }
+                int *z = cnt + (par ^ 1) * sc * 3 + sg * 3;
+                z[0] = 0; z[1] = 0; z[2] = 0;
+            }
+            __syncthreads();
+        }
+    };
+    // Marks the winners of a seg_search among this thread's tokens: keys above the segment's
+    // threshold, and of the keys equal to it the first take_s in position order.
+    // raise_only: only sets flags (backfill); otherwise writes the flag of every active token.
+    auto seg_mark = [&](const int *bnd, unsigned act, int s0, unsigned nsb, bool raise_only) {
+        const bool need_rank = sm.bcast[7] != 0;
+        unsigned keepb = 0, tieb = 0;
+        int my_t = 0;
+        if (act) {
+            int s = s0;
+            unsigned th = cand[s];
+            bool all_ties = takev[s] >= tiesv[s];
+#pragma unroll
+            for (int i = 0; i < VPT; ++i) {
+                if (i > 0 && ((nsb >> i) & 1u)) { ++s; th = cand[s]; all_ties = takev[s] >= tiesv[s]; }
+                if ((act >> i) & 1u) {
+                    const unsigned k = key[i];
+                    if (k > th) keepb |= 1u << i;
+                    else if (k == th) {
+                        if (all_ties) keepb |= 1u << i;
+                        else { tieb |= 1u << i; ++my_t; }
+                    }
+                }
+            }
+        }
+        if (need_rank) { // same decision in every thread of the cluster
+            u64 before_blocks, bt;
+            unit_sum((u64)my_t, &before_blocks);
+            const int run0 = (int)before_blocks + (int)block_excl_scan_u64((u64)my_t, sm.scratch, &bt);
+            auto tp_put = [&](int sg, int v) {
+                if (cs == 1) tps[sg] = v;
+                else for (int r = 0; r < cs; ++r) *cluster.map_shared_rank(tps + sg, r) = v;
+            };
+            if (valid) { // number of tied keys before the first token of each segment
+                int s = s0, run = run0;
+                if (t_base + my0 == bnd[s0]) tp_put(s0, run);
+#pragma unroll
+                for (int i = 0; i < VPT; ++i) {
+                    if (i > 0 && ((nsb >> i) & 1u)) { ++s; tp_put(s, run); }
+                    if ((tieb >> i) & 1u) ++run;
+                }
+            }
+            unit_barrier();
+            if (act) {
+                int s = s0, run = run0, base = tps[s], tk = takev[s];
+#pragma unroll
+                for (int i = 0; i < VPT; ++i) {
+                    if (i > 0 && ((nsb >> i) & 1u)) { ++s; base = tps[s]; tk = takev[s]; }
+                    if ((tieb >> i) & 1u) { if (run - base < tk) keepb |= 1u << i; ++run; }
+                }
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            if ((act >> i) & 1u) {
+                if ((keepb >> i) & 1u) flags[my0 + i] = 1;
+                else if (!raise_only) flags[my0 + i] = 0;
+            }
+        }
+    };
+
+    // ---- per-segment top-q_i by (score desc, position asc)
+    seg_search(quota, n_seg, valid, seg0, newseg);
+    seg_mark(bounds, valid, seg0, newseg, false);
+    unit_barrier();
+
+    // ---- must-keep prefix and suffix; every must-keep position a segment already chose
+    //      frees one slot, refilled by the best positions not yet kept (one pseudo-segment
+    //      [0, T) whose candidates are the tokens without a flag)
+    long long already = 0;
+    for (int i = tid; i < ns + nl; i += nt) {
+        const int t = (i < ns ? i : T - nl + (i - ns)) - t_base;
+        if (t >= 0 && t < n_loc) { already += flags[t]; flags[t] = 1; }
+    }
+    const int r_fill = (int)unit_sum((u64)already, nullptr);
+    if (r_fill > 0) {
+        if (tid == 0) { merged[0] = 0; merged[1] = T; poff[0] = r_fill; }
+        unsigned act = 0;
+#pragma unroll
+        for (int i = 0; i < VPT; ++i)
+            if (((valid >> i) & 1u) && flags[my0 + i] == 0) act |= 1u << i;
+        __syncthreads();
+        seg_search(poff, 1, act, 0, 0u);
+        seg_mark(merged, act, 0, 0u, true);
+    }
+    __syncthreads();
+
+    // ---- ordered compaction of the kept positions; credit rows travel with their tokens
+    //      and rows beyond the budget start from zero
+    unsigned kept_bits = 0;
+    int n_kept = 0;
+#pragma unroll
+    for (int i = 0; i < VPT; ++i)
+        if (my0 + i < n_loc && flags[my0 + i]) { kept_bits |= 1u << i; ++n_kept; }
+    u64 before_blocks, btot3;
+    const int total = (int)unit_sum((u64)n_kept, &before_blocks);
+    int pos = (int)before_blocks + (int)block_excl_scan_u64((u64)n_kept, sm.scratch, &btot3);
+    if (total != p.Tk) {
+        if (tid == 0 && rank == 0) set_status(p.status, AMS_ERR_INTERNAL, uid, total, p.Tk);
+    } else {
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            const int t = t_base + my0 + i;
+            if (kept_bits & (1u << i)) {
+                keep[pos] = t;
+                if (ema_on) credit[pos] = crs[i * nt + tid];
+                ++pos;
+            }
+            if (ema_on && my0 + i < n_loc && t >= p.Tk) credit[t] = 0.0f;
+        }
+    }
+    if (cs > 1) cluster.sync(); // nobody leaves while a neighbour may still read its shared memory
+}
+
+template <int NT, int VPT>
+int launch_cfg(const DevParams &p, LaunchCtx &ctx, int cs, size_t smem)
+{
+    static size_t configured = 0;
+    if (smem > configured) {
+        if (cudaFuncSetAttribute(k_segment_select_cluster<NT, VPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return AMS_ERR_CUDA;
+        configured = smem;
+    }
+    const int units = p.L * p.B * p.H;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3((unsigned)(units * cs), 1, 1);
+    cfg.blockDim = dim3(NT, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = ctx.s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cs;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, k_segment_select_cluster<NT, VPT>, p, cs) != cudaSuccess) return AMS_ERR_CUDA;
+    ctx.mark(kKernSegmentSelect);
+    return AMS_OK;
+}
+
+constexpr int kNT = 1024;
+
+} // namespace
+
+// True when the on-chip kernel can take this call: the sequence capacity fits one cluster of
+// at most eight blocks and the segment tables fit beside the per-token arrays.
+bool segment_cluster_supported(const DevParams &p)
+{
+    if (p.T_cap > 8 * kNT * 16 || p.usage != p.scores) return false;
+    const int vpt = p.T_cap <= kNT * 4 ? 4 : (p.T_cap <= kNT * 8 ? 8 : 16);
+    return smem_map(kNT * vpt, p.seg_cap, p.S, p.beta != 1.0f).total <= (size_t)200 * 1024;
+}
+
+int launch_segment_select_cluster(const DevParams &p, LaunchCtx &ctx)
+{
+    const bool ema_on = p.beta != 1.0f;
+    if (p.T_cap <= kNT * 4) return launch_cfg<kNT, 4>(p, ctx, 1, smem_map(kNT * 4, p.seg_cap, p.S, ema_on).total);
+    if (p.T_cap <= kNT * 8) return launch_cfg<kNT, 8>(p, ctx, 1, smem_map(kNT * 8, p.seg_cap, p.S, ema_on).total);
+    const int tpc = kNT * 16;
+    const int cs_need = (p.T_cap + tpc - 1) / tpc;
+    int cs = 1;
+    while (cs < cs_need) cs *= 2; // cluster sizes are powers of two
+    return launch_cfg<kNT, 16>(p, ctx, cs, smem_map(tpc, p.seg_cap, p.S, ema_on).total);
+}
+
+} // namespace ams

@@ -55,6 +55,15 @@ EXT_CASES = [
     ("lognormal", dict(seq_len_min=1000, seq_len_max=1777, batch=4, budget=1200, n_last=0)),  # ragged; some skipped
     ("lognormal", dict(budget=5, n_sink=4, n_last=16, q_min=2, n_segments=10)),               # budget below minima
     ("ties", dict(seq_len_min=9001, seq_len_max=9001, budget=2048, batch=1, n_layers=1, l_max=4096, n_segments=16)),
+    # sequences that span a cluster of 2 / 4 / 8 blocks
+    ("lognormal", dict(seq_len_min=20011, seq_len_max=20011, budget=3000, batch=1, n_layers=1)),
+    ("ties", dict(seq_len_min=17000, seq_len_max=40000, budget=4096, batch=3, n_layers=1, l_max=4096, n_segments=16)),
+    ("lognormal", dict(seq_len_min=70001, seq_len_max=70001, budget=8192, batch=1, n_layers=1, n_kv_heads=2, n_q_heads=8,
+                       l_max=8192, n_segments=32)),
+    ("ties", dict(seq_len_min=33000, seq_len_max=33000, budget=500, batch=1, n_layers=1, n_segments=1, l_max=0, n_sink=0,
+                  n_last=0, q_min=0, ema_beta=1.0)),                                           # global top-k over 4 blocks
+    ("spike", dict(seq_len_min=50000, seq_len_max=50000, budget=6000, batch=1, n_layers=1, n_kv_heads=2, n_q_heads=8)),
+    ("ties", dict(seq_len_min=3000, seq_len_max=3000, budget=700, l_min=1, l_max=5, n_segments=64, q_min=2)),  # many tiny segments
 ]
 
 
