@@ -431,7 +431,8 @@ __global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, i
         for (int s = tid; s < nsg; s += nt) cand[s] = 0u;
         for (int i = tid; i < nsg * 3; i += nt) { cnt[i] = 0; cnt[sc * 3 + i] = 0; }
         if (tid == 0) sm.bcast[7] = 0;
-        const bool wuni = __all_sync(0xffffffffu, nsb == 0 && s0 == __shfl_sync(0xffffffffu, s0, 0));
+        const int s0_first = __shfl_sync(0xffffffffu, s0, 0); // every lane takes part (no short-circuit around it)
+        const bool wuni = __all_sync(0xffffffffu, nsb == 0 && s0 == s0_first);
         __syncthreads();
         int par = 0;
         for (int shift = 30; shift >= -2; shift -= 2, par ^= 1) {
