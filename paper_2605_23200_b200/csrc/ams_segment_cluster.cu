@@ -12,6 +12,8 @@
 #include <cooperative_groups.h>
 #include <string.h>
 
+#include <type_traits>
+
 #include "ams_common.cuh"
 #include "ams_select.cuh"
 
@@ -65,6 +67,7 @@ __global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, i
     extern __shared__ __align__(16) unsigned char dyn[];
     __shared__ Smem sm;
     __shared__ u64 xch[kXch];
+    __shared__ int wcnt[64]; // per-warp counts of even / odd search rounds
     cg::cluster_group cluster = cg::this_cluster();
     const int tid = threadIdx.x, lane = tid & 31;
     const int rank = cs > 1 ? (int)cluster.block_rank() : 0;
@@ -134,6 +137,18 @@ __global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, i
         float m = mine;
         for (int r = 0; r < cs; ++r) m = fmaxf(m, __uint_as_float((unsigned)*cluster.map_shared_rank(slot, r)));
         return m;
+    };
+
+    // Score / flag of any token of the sequence, wherever it lives in the cluster (a short
+    // segment may straddle two blocks).
+    auto g_at = [&](int t) -> float {
+        const int r = t / TPC;
+        return r == rank ? gs[t - t_base] : *cluster.map_shared_rank(gs + (t - r * TPC), r);
+    };
+    auto flag_put = [&](int t, unsigned char f) {
+        const int r = t / TPC;
+        if (r == rank) flags[t - t_base] = f;
+        else *cluster.map_shared_rank(flags + (t - r * TPC), r) = f;
     };
 
     // ---- scores into shared memory (token order); cut table starts at "no cut"
@@ -559,9 +574,84 @@ __global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, i
         }
     };
 
-    // ---- per-segment top-q_i by (score desc, position asc)
-    seg_search(quota, n_seg, valid, seg0, newseg);
-    seg_mark(bounds, valid, seg0, newseg, false);
+    // ---- per-segment top-q_i by (score desc, position asc).
+    //      Segments of at most 1024 tokens (always, when 0 < l_max <= 1024): one warp per
+    //      segment, in the block that owns the segment's first token, keys in registers; the
+    //      q-th largest key is found bit by bit from the top (count of keys >= prefix | bit,
+    //      one warp reduction per bit) and the search stops as soon as exactly q keys lie at
+    //      or above the prefix.  Otherwise: all segments at once with seg_search.
+    if (p.l_max > 0 && p.l_max <= 1024) {
+        int s_lo, s_hi; // segments whose first token this block owns
+        {
+            int lo = 0, hi = n_seg;
+            while (lo < hi) { const int mid = (lo + hi) >> 1; if (bounds[mid] < t_base) lo = mid + 1; else hi = mid; }
+            s_lo = lo;
+            hi = n_seg;
+            while (lo < hi) { const int mid = (lo + hi) >> 1; if (bounds[mid] < t_base + TPC) lo = mid + 1; else hi = mid; }
+            s_hi = lo;
+        }
+        auto warp_segment = [&](auto kpl_tag, int a, int e, int q) {
+            constexpr int KPL = decltype(kpl_tag)::value;
+            unsigned k[KPL];
+#pragma unroll
+            for (int j = 0; j < KPL; ++j) {
+                const int t = a + j * 32 + lane;
+                k[j] = t < e ? score_key(g_at(t)) : 0u; // keys that are 0 never count below (X >= 1)
+            }
+            unsigned P = 0;
+            bool exact = false;
+            for (int bit = 31; bit >= 0; --bit) {
+                const unsigned X = P | (1u << bit);
+                int c = 0;
+#pragma unroll
+                for (int j = 0; j < KPL; ++j) c += k[j] >= X;
+                c = __reduce_add_sync(0xffffffffu, c);
+                if (c >= q) {
+                    P = X;
+                    if (c == q) { exact = true; break; }
+                }
+            }
+            int take = 0;
+            if (!exact) { // P is the q-th largest key itself; some of the keys equal to it stay out
+                int c = 0;
+#pragma unroll
+                for (int j = 0; j < KPL; ++j) c += k[j] > P;
+                take = q - __reduce_add_sync(0xffffffffu, c);
+            }
+            int seen = 0;
+#pragma unroll
+            for (int j = 0; j < KPL; ++j) {
+                const int t = a + j * 32 + lane;
+                const bool in = t < e;
+                bool keepit = in && k[j] > P;
+                const bool tie = in && k[j] == P;
+                if (exact) keepit |= tie;
+                else {
+                    const unsigned bal = __ballot_sync(0xffffffffu, tie);
+                    keepit |= tie && seen + __popc(bal & ((1u << lane) - 1u)) < take;
+                    seen += __popc(bal);
+                }
+                if (in) flag_put(t, keepit ? 1 : 0);
+            }
+        };
+        const int warp = tid >> 5;
+        for (int s = s_lo + warp; s < s_hi; s += nt / 32) {
+            const int a = bounds[s], e = bounds[s + 1], q = quota[s], L = e - a;
+            if (q <= 0 || q >= L) {
+                const unsigned char f = q >= L ? 1 : 0;
+                for (int t = a + lane; t < e; t += 32) flag_put(t, f);
+            } else if (L <= 256) {
+                warp_segment(std::integral_constant<int, 8>{}, a, e, q);
+            } else if (L <= 512) {
+                warp_segment(std::integral_constant<int, 16>{}, a, e, q);
+            } else {
+                warp_segment(std::integral_constant<int, 32>{}, a, e, q);
+            }
+        }
+    } else {
+        seg_search(quota, n_seg, valid, seg0, newseg);
+        seg_mark(bounds, valid, seg0, newseg, false);
+    }
     unit_barrier();
 
     // ---- must-keep prefix and suffix; every must-keep position a segment already chose
@@ -574,14 +664,65 @@ __global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, i
     }
     const int r_fill = (int)unit_sum((u64)already, nullptr);
     if (r_fill > 0) {
-        if (tid == 0) { merged[0] = 0; merged[1] = T; poff[0] = r_fill; }
+        // Bit-by-bit search for the r_fill-th largest key among the unflagged tokens of the
+        // whole sequence: per round one count per warp, one barrier, and every thread adds up
+        // the warps' (and blocks') counts itself.  Stops once exactly r_fill keys qualify.
         unsigned act = 0;
 #pragma unroll
-        for (int i = 0; i < VPT; ++i)
+        for (int i = 0; i < VPT; ++i) {
             if (((valid >> i) & 1u) && flags[my0 + i] == 0) act |= 1u << i;
-        __syncthreads();
-        seg_search(poff, 1, act, 0, 0u);
-        seg_mark(merged, act, 0, 0u, true);
+            else key[i] = 0u; // never counted (X >= 1)
+        }
+        constexpr int nwarps = nt / 32;
+        int *wc = wcnt;
+        auto unit_count = [&](int c, int n) -> int {
+            c = __reduce_add_sync(0xffffffffu, c);
+            int *mine = wc + (n & 1) * 32;
+            if (lane == 0) mine[tid >> 5] = c;
+            unit_barrier();
+            int v = 0;
+            if (cs == 1) v = lane < nwarps ? mine[lane] : 0;
+            else for (int r = 0; r < cs; ++r) v += lane < nwarps ? cluster.map_shared_rank(mine, r)[lane] : 0;
+            return __reduce_add_sync(0xffffffffu, v);
+        };
+        unsigned P = 0;
+        bool exact = false;
+        int n = 0;
+        for (int bit = 31; bit >= 0; --bit, ++n) {
+            const unsigned X = P | (1u << bit);
+            int c = 0;
+#pragma unroll
+            for (int i = 0; i < VPT; ++i) c += key[i] >= X;
+            const int tot = unit_count(c, n);
+            if (tot >= r_fill) {
+                P = X;
+                if (tot == r_fill) { exact = true; break; }
+            }
+        }
+        unsigned keepb = 0, tieb = 0;
+        int my_t = 0;
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            if ((act >> i) & 1u) {
+                if (key[i] > P || (exact && key[i] == P)) keepb |= 1u << i;
+                else if (key[i] == P) { tieb |= 1u << i; ++my_t; }
+            }
+        }
+        if (!exact) { // the first (r_fill - #keys above P) of the keys equal to P, in position order
+            int c = 0;
+#pragma unroll
+            for (int i = 0; i < VPT; ++i) c += key[i] > P;
+            const int take = r_fill - unit_count(c, n);
+            u64 before_blocks, bt;
+            unit_sum((u64)my_t, &before_blocks);
+            int rk = (int)before_blocks + (int)block_excl_scan_u64((u64)my_t, sm.scratch, &bt);
+#pragma unroll
+            for (int i = 0; i < VPT; ++i)
+                if ((tieb >> i) & 1u) { if (rk < take) keepb |= 1u << i; ++rk; }
+        }
+#pragma unroll
+        for (int i = 0; i < VPT; ++i)
+            if ((keepb >> i) & 1u) flags[my0 + i] = 1;
     }
     __syncthreads();
 
