@@ -16,7 +16,8 @@
  * floating-point operation below is one IEEE-754 round-to-nearest operation (no
  * fused multiply-add) and every sum over tokens that feeds a decision is a sum
  * of 64-bit integers obtained by fixed-point conversion with FIX_BITS = 36
- * fractional bits.  Per token this departs from the real-valued definition by
+ * fractional bits.  A normalisation x / total is evaluated as x * (1 / total),
+ * the reciprocal rounded once per sequence.  Per token this departs from the real-valued definition by
  * less than 2^-36 of the total mass.
  *
  * Pins (see tests, CPU-only): Eq. 1 closed form and sum-to-one; cuts against an
@@ -200,13 +201,16 @@ void orc_weights(const float *u, int32_t T, float eps, float *w)
     }
 }
 
-/* m_t = A_t / sum(A): Eq. 1 on the fixed-point weights, rounded once to fp32. */
+/* m_t = A_t / sum(A): Eq. 1 on the fixed-point weights.  The normalisation is a product
+ * with the reciprocal of the total, rounded once to fp64 (1 / SA), then the product rounded
+ * to fp64 and to fp32: two roundings of 2^-53 against a decision quantum of 2^-36. */
 void orc_mass(const float *u, int32_t T, float eps, uint64_t *A, uint64_t *SA, float *m)
 {
     float *w = (float *)malloc(sizeof(float) * (size_t)T);
     orc_weights(u, T, eps, w);
     orc_fixed_point(w, T, A, SA);
-    for (int t = 0; t < T; ++t) m[t] = (float)((double)A[t] / (double)*SA);
+    const double inv_sa = 1.0 / (double)*SA;
+    for (int t = 0; t < T; ++t) m[t] = (float)((double)A[t] * inv_sa);
     free(w);
 }
 
@@ -223,8 +227,9 @@ void orc_history_mass(const uint64_t *A, uint64_t SA, const float *m, float *cre
                       float lambda, float beta, uint64_t *Hm)
 {
     const double two_f = ldexp(1.0, FIX_BITS);
+    const double inv_sa = 1.0 / (double)SA; /* normalisations multiply by the rounded reciprocal */
     if (beta == 1.0f) {
-        for (int t = 0; t < T; ++t) Hm[t] = (uint64_t)floor(((double)A[t] / (double)SA) * two_f);
+        for (int t = 0; t < T; ++t) Hm[t] = (uint64_t)floor(((double)A[t] * inv_sa) * two_f);
         return;
     }
     const float oml = 1.0f - lambda;
@@ -237,9 +242,10 @@ void orc_history_mass(const uint64_t *A, uint64_t SA, const float *m, float *cre
     uint64_t SC = 0;
     orc_fixed_point(credit, T, Cq, &SC);
     const double bd = (double)beta, omb = 1.0 - (double)beta;
+    const double inv_sc = (SC > 0) ? 1.0 / (double)SC : 0.0;
     for (int t = 0; t < T; ++t) {
-        const double cur = bd * ((double)A[t] / (double)SA);
-        const double hist = (SC > 0) ? omb * ((double)Cq[t] / (double)SC) : 0.0;
+        const double cur = bd * ((double)A[t] * inv_sa);
+        const double hist = (SC > 0) ? omb * ((double)Cq[t] * inv_sc) : 0.0;
         Hm[t] = (uint64_t)floor((cur + hist) * two_f);
     }
     free(Cq);

@@ -57,6 +57,7 @@ __global__ void __launch_bounds__(1024) k_segment_select(DevParams p)
     for (int t = tid; t < T; t += nt) sa += to_fixed(weight_of(u[t], p.eps), sw);
     const u64 SA = block_sum_u64(sa, sm.scratch);
     const double dSA = (double)SA;
+    const double inv_sa = __ddiv_rn(1.0, dSA); // normalisations multiply by the rounded reciprocal of the total
 
     // ---- EMA credit and the mass used for segmentation
     u64 sh = 0;
@@ -65,7 +66,7 @@ __global__ void __launch_bounds__(1024) k_segment_select(DevParams p)
         float cmax = 0.0f;
         for (int t = tid; t < T; t += nt) {
             const u64 A = to_fixed(weight_of(u[t], p.eps), sw);
-            const float m = __double2float_rn(__ddiv_rn((double)A, dSA));
+            const float m = __double2float_rn(__dmul_rn((double)A, inv_sa));
             const float cn = __fadd_rn(__fmul_rn(p.lambda, credit[t]), __fmul_rn(oml, m));
             credit[t] = cn;
             if (mass_dbg) mass_dbg[t] = m;
@@ -80,11 +81,12 @@ __global__ void __launch_bounds__(1024) k_segment_select(DevParams p)
         }
         const u64 SC = block_sum_u64(scsum, sm.scratch);
         const double dSC = (double)SC, bd = (double)p.beta, omb = __dsub_rn(1.0, (double)p.beta);
+        const double inv_sc = SC > 0 ? __ddiv_rn(1.0, dSC) : 0.0;
         for (int t = tid; t < T; t += nt) {
             const u64 A = to_fixed(weight_of(u[t], p.eps), sw);
-            const double cur = __dmul_rn(bd, __ddiv_rn((double)A, dSA));
+            const double cur = __dmul_rn(bd, __dmul_rn((double)A, inv_sa));
             double hist_term = 0.0;
-            if (SC > 0) hist_term = __dmul_rn(omb, __ddiv_rn((double)to_fixed(credit[t], scl), dSC));
+            if (SC > 0) hist_term = __dmul_rn(omb, __dmul_rn((double)to_fixed(credit[t], scl), inv_sc));
             const u64 Hm = (u64)__double2ull_rd(__dmul_rn(__dadd_rn(cur, hist_term), two_f));
             Cb[t] = Hm;
             sh += Hm;
@@ -92,7 +94,7 @@ __global__ void __launch_bounds__(1024) k_segment_select(DevParams p)
     } else {
         for (int t = tid; t < T; t += nt) {
             const u64 A = to_fixed(weight_of(u[t], p.eps), sw);
-            const double r = __ddiv_rn((double)A, dSA);
+            const double r = __dmul_rn((double)A, inv_sa);
             if (mass_dbg) mass_dbg[t] = __double2float_rn(r);
             const u64 Hm = (u64)__double2ull_rd(__dmul_rn(r, two_f));
             Cb[t] = Hm;

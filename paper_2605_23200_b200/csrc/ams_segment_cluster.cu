@@ -189,16 +189,16 @@ __global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, i
         for (int i = 0; i < VPT; ++i) wmax = fmaxf(wmax, w[i]);
     }
     wmax = unit_max(wmax);
-    const double sw = fix_scale(wmax);
+    const int ew = fix_exponent(wmax);
     u64 sa = 0;
     {
         float w[VPT];
         load_w(w);
 #pragma unroll
-        for (int i = 0; i < VPT; ++i) sa += to_fixed(w[i], sw);
+        for (int i = 0; i < VPT; ++i) sa += to_fixed_bits(w[i], ew);
     }
     const u64 SA = unit_sum(sa, nullptr);
-    const double dSA = (double)SA;
+    const double inv_sa = __ddiv_rn(1.0, (double)SA); // normalisations multiply by the rounded reciprocal
 
     // ---- EMA credit and the fixed-point mass used for segmentation
     float *mass_dbg = p.mass_dbg ? p.mass_dbg + row + t_base + my0 : nullptr;
@@ -211,8 +211,7 @@ __global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, i
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
             if (my0 + i < n_loc) {
-                const u64 A = to_fixed(w[i], sw);
-                const float m = __double2float_rn(__ddiv_rn((double)A, dSA));
+                const float m = __double2float_rn(__dmul_rn(u52_to_double(to_fixed_bits(w[i], ew)), inv_sa));
                 const float cn = __fadd_rn(__fmul_rn(p.lambda, crs[i * nt + tid]), __fmul_rn(oml, m));
                 crs[i * nt + tid] = cn;
                 if (mass_dbg) mass_dbg[i] = m;
@@ -221,25 +220,24 @@ __global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, i
         }
         cmax = unit_max(cmax);
         u64 scsum = 0;
-        double scl = 0.0;
+        int ec = 0;
         if (cmax > 0.0f) {
-            scl = fix_scale(cmax);
+            ec = fix_exponent(cmax);
 #pragma unroll
             for (int i = 0; i < VPT; ++i)
-                if (my0 + i < n_loc) scsum += to_fixed(crs[i * nt + tid], scl);
+                if (my0 + i < n_loc) scsum += to_fixed_bits(crs[i * nt + tid], ec);
         }
         const u64 SC = unit_sum(scsum, nullptr);
-        const double dSC = (double)SC, bd = (double)p.beta, omb = __dsub_rn(1.0, (double)p.beta);
-        load_w(w);
+        const double bd = (double)p.beta, omb = __dsub_rn(1.0, (double)p.beta);
+        const double inv_sc = SC > 0 ? __ddiv_rn(1.0, (double)SC) : 0.0;
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
             Hm[i] = 0;
             if (my0 + i < n_loc) {
-                const u64 A = to_fixed(w[i], sw);
-                const double cur = __dmul_rn(bd, __ddiv_rn((double)A, dSA));
+                const double cur = __dmul_rn(bd, __dmul_rn(u52_to_double(to_fixed_bits(w[i], ew)), inv_sa));
                 double hist_term = 0.0;
-                if (SC > 0) hist_term = __dmul_rn(omb, __ddiv_rn((double)to_fixed(crs[i * nt + tid], scl), dSC));
-                Hm[i] = (u64)__double2ull_rd(__dmul_rn(__dadd_rn(cur, hist_term), two_f));
+                if (SC > 0) hist_term = __dmul_rn(omb, __dmul_rn(u52_to_double(to_fixed_bits(crs[i * nt + tid], ec)), inv_sc));
+                Hm[i] = floor_to_u64(__dmul_rn(__dadd_rn(cur, hist_term), two_f));
             }
         }
     } else {
@@ -249,10 +247,9 @@ __global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, i
         for (int i = 0; i < VPT; ++i) {
             Hm[i] = 0;
             if (my0 + i < n_loc) {
-                const u64 A = to_fixed(w[i], sw);
-                const double r = __ddiv_rn((double)A, dSA);
+                const double r = __dmul_rn(u52_to_double(to_fixed_bits(w[i], ew)), inv_sa);
                 if (mass_dbg) mass_dbg[i] = __double2float_rn(r);
-                Hm[i] = (u64)__double2ull_rd(__dmul_rn(r, two_f));
+                Hm[i] = floor_to_u64(__dmul_rn(r, two_f));
             }
         }
     }

@@ -166,5 +166,36 @@ __device__ void radix_select(const float *g, int a, int b, int k, int *hist, int
     *ties = n_ties;
 }
 
+// ---- the same fixed-point images without 64-bit conversions -------------------------------
+// Exponent e = ilogb(mx) + 1 of the largest weight mx > 0 (any fp32, subnormals included).
+__device__ __forceinline__ int fix_exponent(float mx)
+{
+    const long long bits = __double_as_longlong((double)mx);
+    return (int)((bits >> 52) & 0x7ff) - 1023 + 1;
+}
+
+// floor(x * 2^(kFixBits - e)) for 0 <= x < 2^e, from the bits of x: x = m * 2^(E - 23) with a
+// 24-bit integer m, so the image is m shifted by E + 13 - e (at most 12 to the left).
+__device__ __forceinline__ u64 to_fixed_bits(float x, int e)
+{
+    const unsigned b = __float_as_uint(x);
+    const int ef = (int)((b >> 23) & 0xffu);
+    const u64 m = ef ? ((b & 0x7fffffu) | 0x800000u) : (b & 0x7fffffu);
+    const int sh = (ef ? ef - 127 : -126) + (kFixBits - 23) - e;
+    return sh >= 0 ? (m << sh) : (sh > -24 ? (m >> (-sh)) : 0ull);
+}
+
+// (double)a for an integer a < 2^52, exact.
+__device__ __forceinline__ double u52_to_double(u64 a)
+{
+    return __dsub_rn(__longlong_as_double((long long)(0x4330000000000000ull | a)), 4503599627370496.0);
+}
+
+// floor(y) for 0 <= y < 2^51 as an integer: y + 2^52 rounded down lands on the integer grid.
+__device__ __forceinline__ u64 floor_to_u64(double y)
+{
+    return (u64)__double_as_longlong(__dadd_rd(y, 4503599627370496.0)) & 0xfffffffffffffull;
+}
+
 } // namespace sel
 } // namespace ams
