@@ -4,7 +4,7 @@
 // Work is the concatenation of all units' 128-token tiles; block c of a persistent grid
 // takes the contiguous tile range [c * tpc, (c + 1) * tpc).  Inside a block:
 //   warp 0      TMA producer: query block of the current unit, then one 32 KB K tile per
-//               stage (eight 16-token pages, two 64-wide halves each, 128-byte swizzle);
+//               stage (eight 16-token pages, one 4 KB copy each, 128-byte swizzle);
 //   warp 1      MMA issuer (one lane): per (tile, 128-row query block) eight
 //               tcgen05.mma m128 n128 k16 into one of four 128-column TMEM slots (two per
 //               consumer warpgroup, used in turn);
@@ -29,7 +29,7 @@ constexpr int kTileTokens = 128;
 constexpr int kTileBytes = kTileTokens * kRowBytes;  // 32 KB
 constexpr int kHalfBytes = kTileBytes / 2;           // one 64-wide half of a 128-row tile
 constexpr int kSlots = 4;                            // TMEM accumulator slots of 128 columns
-constexpr int kMaxStages = 4;
+constexpr int kMaxStages = 6;
 constexpr uint32_t kWaitLimit = 1u << 22;
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -112,10 +112,10 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, unsigned long long a_des
     asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
                  ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
-// 32 consecutive fp32 columns of this thread's TMEM lane.
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32])
+// 32 consecutive fp32 columns of this thread's TMEM lane, asynchronously: the registers
+// are valid only after tc_ld_wait on the same array.
+__device__ __forceinline__ void tc_ld32_issue(uint32_t taddr, uint32_t (&r)[32])
 {
-    uint32_t r[32];
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
                  "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
@@ -123,16 +123,31 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32])
                    "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
                    "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
                  : "r"(taddr) : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+// Waits for every tcgen05.ld this thread has issued; the array is named as an in/out operand
+// so that no use of it is scheduled above the wait.
+__device__ __forceinline__ void tc_ld_wait(uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                   "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                   "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+                   "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+                 :: "memory");
+}
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
 }
 
 // Shared-memory matrix descriptor of a K-major, 128-byte-swizzled tile whose rows are
-// 128 bytes (64 bf16) and whose 8-row groups are 1024 bytes apart.
-__device__ __forceinline__ unsigned long long smem_desc(uint32_t addr)
+// 128 bytes (64 bf16) and whose 8-row groups are `group_stride` bytes apart.
+__device__ __forceinline__ unsigned long long smem_desc(uint32_t addr, uint32_t group_stride)
 {
-    return (unsigned long long)((addr & 0x3ffffu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+    return (unsigned long long)((addr & 0x3ffffu) >> 4) | (1ull << 16) | ((unsigned long long)(group_stride >> 4) << 32) | (1ull << 46) |
+           (2ull << 61);
 }
 // kind::f16 instruction descriptor: fp32 accumulate, bf16 x bf16, both K-major, M = N = 128.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
@@ -143,7 +158,10 @@ __device__ __forceinline__ int tiles_of(const DevParams &p, int b)
     return (T > p.Tk && T <= p.T_cap && p.W <= T) ? (T + kTileTokens - 1) / kTileTokens : 0;
 }
 
-// Prefix of tiles per sequence (shared by all layers and heads) and the block partition.
+// Prefix of tiles per sequence (shared by all layers and heads) and the partition of one head's
+// tiles (all layers) over `grid` groups of blocks.  A group is H blocks, one per KV head, that
+// walk the same token tiles at the same time: together they read whole pages (all heads of
+// 16 tokens are contiguous), which DRAM serves far better than one head's 256-byte rows alone.
 __device__ void tc_partition(const DevParams &p, int grid, int *prefix, int *tiles_lh, long long *n_tiles, int *tpc)
 {
     if (threadIdx.x == 0) {
@@ -151,7 +169,7 @@ __device__ void tc_partition(const DevParams &p, int grid, int *prefix, int *til
         for (int b = 0; b < p.B; ++b) { prefix[b] = acc; acc += tiles_of(p, b); }
         prefix[p.B] = acc;
         *tiles_lh = acc;
-        const long long N = (long long)p.L * p.H * acc;
+        const long long N = (long long)p.L * acc;
         *n_tiles = N;
         const long long per = (N + grid - 1) / grid;
         *tpc = (int)(per > p.tc_tpc_min ? per : p.tc_tpc_min);
@@ -162,13 +180,13 @@ __device__ void tc_partition(const DevParams &p, int grid, int *prefix, int *til
 struct Segment { int uid, l, b, h, tile0, n, T, part; };
 
 // Decodes the segment that starts at global tile g and ends no later than `end`.
-__device__ __forceinline__ Segment decode_segment(const DevParams &p, const int *prefix, int tiles_lh, int tpc, long long g, long long end)
+__device__ __forceinline__ Segment decode_segment(const DevParams &p, const int *prefix, int tiles_lh, int tpc, long long g, long long end, int h)
 {
     Segment s;
-    const int lh = (int)(g / tiles_lh), rem = (int)(g % tiles_lh);
+    const int l = (int)(g / tiles_lh), rem = (int)(g % tiles_lh);
     int b = 0;
     while (prefix[b + 1] <= rem) ++b;
-    s.l = lh / p.H; s.h = lh % p.H; s.b = b;
+    s.l = l; s.h = h; s.b = b;
     s.uid = (s.l * p.B + b) * p.H + s.h;
     s.tile0 = rem - prefix[b];
     const int left = prefix[b + 1] - rem;
@@ -205,7 +223,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    tc_partition(p, gridDim.x, prefix, &sh.tiles_lh, &sh.n_tiles, &sh.tpc);
+    const int my_h = blockIdx.x % p.H, my_group = blockIdx.x / p.H;
+    tc_partition(p, gridDim.x / p.H, prefix, &sh.tiles_lh, &sh.n_tiles, &sh.tpc);
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)), "r"(512) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -215,7 +234,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
     tc_fence_after();
     const uint32_t tmem_base = sh.tmem_base;
     const int tiles_lh = sh.tiles_lh, tpc = sh.tpc;
-    const long long g_begin = (long long)blockIdx.x * tpc;
+    const long long g_begin = (long long)my_group * tpc;
     const long long g_end = (g_begin + tpc < sh.n_tiles) ? g_begin + tpc : sh.n_tiles;
     if (PHASE == 1 && blockIdx.x == 0 && tid == 0) {
         for (int b = 0; b < p.B; ++b) {
@@ -231,7 +250,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
             int kit = 0, seg = 0, issued = 0;
             bool ok = true;
             for (long long g = g_begin; g < g_end && ok;) {
-                const Segment s = decode_segment(p, prefix, tiles_lh, tpc, g, g_end);
+                const Segment s = decode_segment(p, prefix, tiles_lh, tpc, g, g_end, my_h);
                 ok = mbar_wait(smem_u32(&sh.qempty), (uint32_t)((seg & 1) ^ 1), abort_flag);
                 if (!ok) break;
                 if (lane == 0) {
@@ -250,12 +269,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
                     if (!ok) break;
                     if (lane == 0) mbar_expect_tx(smem_u32(&sh.kfull[st]), (uint32_t)kTileBytes);
                     __syncwarp();
-                    if (lane < 16) {
-                        const int pg = lane >> 1, hf = lane & 1;
+                    if (lane < 8) {
+                        // one copy per page: both 64-wide halves of this head's 16 rows (4 KB)
+                        const int pg = lane;
                         int pi = (s.tile0 + i) * 8 + pg;
                         if (pi > last_page) pi = last_page;  // tokens past the end are masked by position
-                        tma_load_5d(smem_u32(Ks + (size_t)st * kTileBytes + hf * kHalfBytes + pg * 2048), &k_map,
-                                    smem_u32(&sh.kfull[st]), hf * 64, s.h, 0, table[pi], s.l);
+                        tma_load_5d(smem_u32(Ks + (size_t)st * kTileBytes + pg * 4096), &k_map, smem_u32(&sh.kfull[st]), 0, 0, 2 * s.h, 0,
+                                    s.l * (int)p.num_pages + table[pi]);
                     }
                     issued = kit + 1;
                 }
@@ -275,7 +295,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
                 int wsit[2] = {0, 0}; // accumulator slots handed to each consumer warpgroup so far
                 bool ok = true;
                 for (long long g = g_begin; g < g_end && ok;) {
-                    const Segment s = decode_segment(p, prefix, tiles_lh, tpc, g, g_end);
+                    const Segment s = decode_segment(p, prefix, tiles_lh, tpc, g, g_end, my_h);
                     ok = mbar_wait(smem_u32(&sh.qfull), (uint32_t)(seg & 1), abort_flag);
                     for (int i = 0; i < s.n && ok; ++i, ++kit) {
                         const int st = kit % NS;
@@ -290,8 +310,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
                             const uint32_t qa = smem_u32(Qs + (size_t)rb * kTileBytes), ka = smem_u32(Ks + (size_t)st * kTileBytes);
 #pragma unroll
                             for (int k = 0; k < 8; ++k) {
-                                const uint32_t off = (uint32_t)((k >> 2) * kHalfBytes + (k & 3) * 32);
-                                const unsigned long long dq = smem_desc(qa + off), dk = smem_desc(ka + off);
+                                // Q tile: [half][128 rows][128 B]; K tile: [8-row group][half][8 rows][128 B]
+                                const unsigned long long dq = smem_desc(qa + (uint32_t)((k >> 2) * kHalfBytes + (k & 3) * 32), 1024);
+                                const unsigned long long dk = smem_desc(ka + (uint32_t)((k >> 2) * 1024 + (k & 3) * 32), 2048);
                                 tc_mma(tmem_base + (uint32_t)(slot * 128), PHASE == 1 ? dq : dk, PHASE == 1 ? dk : dq, kIdesc, k > 0);
                             }
                             tc_commit(smem_u32(&sh.tfull[slot]));
@@ -316,7 +337,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
             // a thread whose wait ran out keeps walking the segments without touching the pipeline, so that
             // the consumers' named barriers stay matched
             for (long long g = g_begin; g < g_end;) {
-                const Segment s = decode_segment(p, prefix, tiles_lh, tpc, g, g_end);
+                const Segment s = decode_segment(p, prefix, tiles_lh, tpc, g, g_end, my_h);
                 const int T = s.T;
                 float m[4], z[4];
                 int lastv[4];
@@ -345,52 +366,74 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
                         if (!ok) break;
                         tc_fence_after();
                         const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * 128);
+                        // chunks of 32 columns, the load of the next chunk in flight while this one is worked on
+                        uint32_t buf[2][32];
+                        tc_ld32_issue(taddr, buf[0]);
+                        tc_ld_wait(buf[0]);
                         if (PHASE == 1) {
                             const int lv = min(lastv[rb], T - 1);
                             float mr = m[rb], zr = z[rb];
-#pragma unroll 1
+#pragma unroll
                             for (int ch = 0; ch < 4; ++ch) {
-                                float v[32];
-                                tc_ld32(taddr + ch * 32, v);
+                                uint32_t (&cur)[32] = buf[ch & 1];
+                                if (ch < 3) tc_ld32_issue(taddr + (ch + 1) * 32, buf[(ch + 1) & 1]);
                                 const int tc0 = t0 + ch * 32;
-                                if (tc0 > lv) continue;
-                                if (tc0 + 31 > lv) {
+                                if (tc0 <= lv) {
+                                    float v[32];
 #pragma unroll
-                                    for (int j = 0; j < 32; ++j) if (tc0 + j > lv) v[j] = -INFINITY;
+                                    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(cur[j]);
+                                    if (tc0 + 31 > lv) {
+#pragma unroll
+                                        for (int j = 0; j < 32; ++j) if (tc0 + j > lv) v[j] = -INFINITY;
+                                    }
+                                    // tree of three-input maxima: depth 4 instead of a chain of 31
+                                    float a8[8];
+#pragma unroll
+                                    for (int j = 0; j < 8; ++j) a8[j] = max3(v[j], v[j + 8], v[j + 16]);
+#pragma unroll
+                                    for (int j = 0; j < 8; ++j) a8[j] = fmaxf(a8[j], v[j + 24]);
+                                    const float cm = fmaxf(max3(a8[0], a8[1], a8[2]), fmaxf(max3(a8[3], a8[4], a8[5]), fmaxf(a8[6], a8[7])));
+                                    const float mn = fmaxf(mr, cm * c);
+                                    zr *= ex2(mr - mn);
+                                    mr = mn;
+                                    float zs[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+                                    for (int j = 0; j < 32; ++j) zs[j & 3] += ex2(fmaf(v[j], c, -mn));
+                                    zr += (zs[0] + zs[1]) + (zs[2] + zs[3]);
                                 }
-                                float cm = v[0];
-#pragma unroll
-                                for (int j = 1; j < 32; ++j) cm = fmaxf(cm, v[j]);
-                                const float mn = fmaxf(mr, cm * c);
-                                zr *= ex2(mr - mn);
-                                mr = mn;
-                                float zs = 0.0f;
-#pragma unroll
-                                for (int j = 0; j < 32; ++j) zs += ex2(fmaf(v[j], c, -mn));
-                                zr += zs;
+                                if (ch < 3) tc_ld_wait(buf[(ch + 1) & 1]);
                             }
                             m[rb] = mr; z[rb] = zr;
                         } else {
                             const int t = t0 + li;
                             const bool plain = !p.causal || t0 + kTileTokens - 1 <= T - p.W;
-                            const float *fr = fs + rb * 128;
-#pragma unroll 1
+                            const float4 *fr4 = reinterpret_cast<const float4 *>(fs + rb * 128);
+                            float ac[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
                             for (int ch = 0; ch < 4; ++ch) {
-                                float v[32];
-                                tc_ld32(taddr + ch * 32, v);
+                                uint32_t (&cur)[32] = buf[ch & 1];
+                                if (ch < 3) tc_ld32_issue(taddr + (ch + 1) * 32, buf[(ch + 1) & 1]);
                                 if (plain) {
 #pragma unroll
-                                    for (int j = 0; j < 32; ++j) acc += ex2(fmaf(v[j], c, -fr[ch * 32 + j]));
+                                    for (int j4 = 0; j4 < 8; ++j4) {
+                                        const float4 f = fr4[ch * 8 + j4];
+                                        ac[0] += ex2(fmaf(__uint_as_float(cur[4 * j4]), c, -f.x));
+                                        ac[1] += ex2(fmaf(__uint_as_float(cur[4 * j4 + 1]), c, -f.y));
+                                        ac[2] += ex2(fmaf(__uint_as_float(cur[4 * j4 + 2]), c, -f.z));
+                                        ac[3] += ex2(fmaf(__uint_as_float(cur[4 * j4 + 3]), c, -f.w));
+                                    }
                                 } else {
                                     const int rbase = rb * 128 + ch * 32;
 #pragma unroll
                                     for (int j = 0; j < 32; ++j) {
                                         const int r = rbase + j;
                                         const bool seen = t <= T - p.W + (r % p.W);
-                                        acc += seen ? ex2(fmaf(v[j], c, -fr[ch * 32 + j])) : 0.0f;
+                                        ac[j & 3] += seen ? ex2(fmaf(__uint_as_float(cur[j]), c, -fs[r])) : 0.0f;
                                     }
                                 }
+                                if (ch < 3) tc_ld_wait(buf[(ch + 1) & 1]);
                             }
+                            acc += (ac[0] + ac[1]) + (ac[2] + ac[3]);
                         }
                         tc_fence_before();
                         __syncwarp();
@@ -442,10 +485,10 @@ __global__ void __launch_bounds__(128) k_tova_combine_tc(DevParams p, int tc_gri
     __shared__ long long s_n;
     tc_partition(p, tc_grid, prefix, &s_tiles_lh, &s_n, &s_tpc);
     const int uid = blockIdx.x;
-    const int h = uid % p.H, b = (uid / p.H) % p.B, l = uid / (p.H * p.B);
+    const int b = (uid / p.H) % p.B, l = uid / (p.H * p.B);
     const int nt = prefix[b + 1] - prefix[b];
     if (nt == 0) return;
-    const long long ustart = (long long)(l * p.H + h) * s_tiles_lh + prefix[b];
+    const long long ustart = (long long)l * s_tiles_lh + prefix[b];
     const int n_parts = (int)((ustart + nt - 1) / s_tpc) - (int)(ustart / s_tpc) + 1;
     float *fin = p.fin + (size_t)uid * (p.rows_pad + 8);
     float best = 0.0f;
@@ -485,7 +528,7 @@ EncodeTiledFn encode_fn()
 
 } // namespace
 
-bool tova_tc_supported(const DevParams &p) { return p.rows >= 64 && p.rows_pad % 128 == 0 && p.rows_pad <= 512 && p.B <= 1024; }
+bool tova_tc_supported(const DevParams &p) { return p.rows >= 64 && p.rows_pad % 128 == 0 && p.rows_pad <= 512 && p.B <= 1024 && p.H <= 64; }
 
 size_t tova_tc_smem_bytes(const DevParams &p)
 {
@@ -499,10 +542,14 @@ int launch_score_tova_tc(const DevParams &p, LaunchCtx &ctx)
     if (!enc) return AMS_ERR_CUDA;
     CUtensorMap k_map, q_map;
     {
-        const cuuint64_t dims[5] = {kHeadDim, (cuuint64_t)p.H, kPage, (cuuint64_t)p.num_pages, (cuuint64_t)p.L};
-        const cuuint64_t strides[4] = {kRowBytes, (cuuint64_t)p.H * kRowBytes, (cuuint64_t)kPage * p.H * kRowBytes,
-                                       (cuuint64_t)p.num_pages * kPage * p.H * kRowBytes};
-        const cuuint32_t box[5] = {64, 1, kPage, 1, 1};
+        // One page of one layer is [16 slots][H heads][2 halves][64]: seen as
+        // (64, slot % 8, head * 2 + half, slot / 8, layer * num_pages + page), so that a box of
+        // (64, 8, 2, 2, 1) is this head's 16 rows, stored as [slot / 8][half][slot % 8][64].
+        if ((long long)p.L * p.num_pages > 0x7fffffffLL) return AMS_ERR_UNSUPPORTED;
+        const cuuint64_t dims[5] = {64, 8, (cuuint64_t)2 * p.H, 2, (cuuint64_t)p.L * (cuuint64_t)p.num_pages};
+        const cuuint64_t strides[4] = {(cuuint64_t)p.H * kRowBytes, 128, (cuuint64_t)8 * p.H * kRowBytes,
+                                       (cuuint64_t)kPage * p.H * kRowBytes};
+        const cuuint32_t box[5] = {64, 8, 2, 2, 1};
         const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
         if (enc(&k_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, p.k_pages, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                 CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
@@ -531,12 +578,14 @@ int launch_score_tova_tc(const DevParams &p, LaunchCtx &ctx)
             return AMS_ERR_CUDA;
         configured = smem;
     }
-    const long long cap_tiles = (long long)p.L * p.B * p.H * ((p.T_cap + kTileTokens - 1) / kTileTokens);
+    const long long cap_tiles = (long long)p.L * p.B * ((p.T_cap + kTileTokens - 1) / kTileTokens); // per head
     long long want = (cap_tiles + p.tc_tpc_min - 1) / p.tc_tpc_min;
-    const int grid = (int)(want < n_sm ? (want < 1 ? 1 : want) : n_sm);
+    const int max_groups = n_sm / p.H;
+    const int groups = (int)(want < max_groups ? (want < 1 ? 1 : want) : max_groups);
+    const int grid = groups * p.H;
     k_tova_tc<1><<<grid, kTcThreads, smem, ctx.s>>>(p, k_map, q_map);
     ctx.mark(kKernScore1);
-    k_tova_combine_tc<<<p.L * p.B * p.H, 128, 0, ctx.s>>>(p, grid);
+    k_tova_combine_tc<<<p.L * p.B * p.H, 128, 0, ctx.s>>>(p, groups);
     ctx.mark(kKernScoreCombine);
     k_tova_tc<2><<<grid, kTcThreads, smem, ctx.s>>>(p, k_map, q_map);
     ctx.mark(kKernScore2);
