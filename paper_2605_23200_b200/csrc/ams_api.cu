@@ -8,7 +8,7 @@
 namespace ams {
 
 struct Layout {
-    size_t status, scores, cbuf, flags, n_seg, seg_bounds, quotas, keep_idx, part, fin, total;
+    size_t status, scores, cbuf, flags, n_seg, seg_bounds, quotas, keep_idx, part, fin, ctrl, finz, total;
     int units, T_cap, seg_cap, n_slices, slice_len, rows_pad_cap;
 };
 
@@ -77,6 +77,9 @@ static Layout make_layout(const ams_config *c)
     if (tc_parts > y.n_slices) y.n_slices = tc_parts;
     const int rows_cap = (c->n_q_heads / c->n_kv_heads) * (c->max_window > 0 ? c->max_window : 1);
     y.rows_pad_cap = rows_padded(rows_cap);
+    // single-pass scorer (query rows padded to 128, sequences of at most 148 tiles): one partial per 128-token tile
+    const int tiles_cap = (y.T_cap + 127) / 128;
+    if (rows_cap >= 64 && y.rows_pad_cap >= 128 && tiles_cap <= 148 && tiles_cap > y.n_slices) y.n_slices = tiles_cap;
     const size_t U = (size_t)y.units, T = (size_t)y.T_cap;
     size_t off = 0;
     y.status = off;     off = align_up(off + 64, 256);
@@ -91,6 +94,8 @@ static Layout make_layout(const ams_config *c)
     y.part = off;       off = align_up(off + U * part_per, 256);
     const size_t fin_per = (size_t)((y.rows_pad_cap > kHeadDim ? y.rows_pad_cap : kHeadDim) + 8) * 4;
     y.fin = off;        off = align_up(off + U * fin_per, 256);
+    y.ctrl = off;       off = align_up(off + U * 2 * 4, 256);
+    y.finz = off;       off = align_up(off + U * 128 * 4, 256);
     y.total = off;
     return y;
 }
@@ -165,6 +170,7 @@ int ams_init_state(const ams_config *cfg, void *ema_state, void *workspace, size
     cudaStream_t s = (cudaStream_t)stream;
     if (cudaMemsetAsync(ema_state, 0, ams_ema_state_bytes(cfg), s) != cudaSuccess) return AMS_ERR_CUDA;
     if (cudaMemsetAsync(workspace, 0, 256, s) != cudaSuccess) return AMS_ERR_CUDA;
+    if (cudaMemsetAsync((unsigned char *)workspace + lay.ctrl, 0, lay.total - lay.ctrl, s) != cudaSuccess) return AMS_ERR_CUDA;
     ams_state *st = new (std::nothrow) ams_state;
     if (!st) return AMS_ERR_INTERNAL;
     st->cfg = *cfg;
@@ -225,6 +231,9 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
     p.tc_tpc_min = tc_tiles_per_block_min(y.T_cap);
     p.tc_stages = p.rows_pad <= 128 ? 4 : (p.rows_pad <= 256 ? 3 : 2);
     p.status = (int *)(st->ws + y.status);
+    p.fcnt = (int *)(st->ws + y.ctrl);
+    p.fflag = p.fcnt + (size_t)c.n_layers * c.max_batch * c.n_kv_heads;
+    p.finz = (float *)(st->ws + y.finz);
 
     int rc = AMS_OK;
     LaunchCtx ctx;

@@ -47,6 +47,8 @@ struct DevParams {
     float *fin;                       // per unit finals
     int slice_len, n_slices, rows_pad;
     int tc_tpc_min, tc_stages;        // tensor-core scorer: least tiles per block, K stages in shared memory
+    int *fcnt, *fflag;                // fused scorer: per-unit counters of tiles in / of query rows merged ([2][units], contiguous)
+    float *finz;                      // fused scorer: 1 / Z_r per unit and query row, [units][rows_pad]
     int *status;                      // [4]: code, unit, a, b
 };
 
@@ -194,6 +196,8 @@ int launch_score_tova(const DevParams &p, LaunchCtx &ctx);
 bool tova_tc_supported(const DevParams &p);
 size_t tova_tc_smem_bytes(const DevParams &p);
 int launch_score_tova_tc(const DevParams &p, LaunchCtx &ctx);
+bool tova_fused_supported(const DevParams &p);
+int launch_score_tova_fused(const DevParams &p, LaunchCtx &ctx);
 int launch_score_keydiff(const DevParams &p, LaunchCtx &ctx);
 int launch_segment_select(const DevParams &p, LaunchCtx &ctx);
 bool segment_cluster_supported(const DevParams &p);
