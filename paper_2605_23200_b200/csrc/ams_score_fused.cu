@@ -20,6 +20,7 @@
 // others waiting for their unit's statistics.  Every wait is bounded; on expiry the block
 // reports AMS_ERR_TIMEOUT and leaves cleanly.
 #include <cuda.h>
+#include <stdlib.h>
 
 #include "ams_common.cuh"
 #include "ams_tc_ptx.cuh"
@@ -417,8 +418,14 @@ size_t fused_smem_bytes() { return 1024 + (size_t)(kQStages + kKStages) * kTileB
 
 } // namespace
 
+// The single-pass scorer is opt-in (environment variable AMS_FUSED_SCORER=1): on B200 the
+// hand-off of the per-tile statistics between blocks (publish, wait for the slowest block,
+// merge) takes longer than the two items of look-ahead that TMEM's 512 columns allow, so the
+// two-kernel scorer, which reads K twice, is the faster one at the benchmark sizes.
 bool tova_fused_supported(const DevParams &p)
 {
+    const char *env = getenv("AMS_FUSED_SCORER");
+    if (!env || env[0] != '1') return false;
     static int n_sm = 0;
     if (!n_sm) {
         int dev = 0;
