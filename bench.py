@@ -44,6 +44,17 @@ def _peaks():
     return 6650.0, "fallback"
 
 
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the scorer passes on the
+# default workload, from the ncu capture summarised in profiles/kernels_cfg1_8layers_ncu_full.md: taken on
+# the 8-layer reduction of the workload and scaled x4 to the 32-layer launch (units are independent and each
+# is read once per pass).  Valid for that workload and the kernels as profiled; anything else reports null.
+NCU_TRAFFIC_BYTES = {
+    "cfg1_llama8b_L32_T16384_k2048_w32": {"score_phase1": 4 * (272_119_296 + 5_242_368),
+                                          "score_phase2": 4 * (272_169_728 + 6_017_536),
+                                          "gather": None},
+}
+
+
 def algorithmic_bytes(wl, lens) -> tuple[int, int]:
     """(K bytes read once for scoring, kept K/V bytes read + written) per step."""
     units = wl.layers_resident * wl.n_kv_heads
@@ -227,7 +238,8 @@ def run_ours(args, rank, world, local_rank):
     out = {
         "metric": METRIC, "value": world * args.steps / (total_ms / 1e3), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16 K/V, fp32 scores, u64 fixed-point decisions",
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "dtype_detail": "bf16 K/V and queries, fp32 accumulation and scores, u64 fixed-point decisions",
         "data": "synthetic",
         "config": {"workload": wl.name, "layers": wl.n_layers, "q_heads": wl.n_q_heads, "kv_heads": wl.n_kv_heads,
                    "batch_per_gpu": wl.batch, "cache_tokens": wl.seq_len_max, "budget": wl.budget, "window": wl.window,
@@ -242,7 +254,9 @@ def run_ours(args, rank, world, local_rank):
         "kernels_ms": kern_ms,
         "roofline": {"kernel": dominant, "bound": "hbm", "achieved": dom_bytes / (dom_ms * 1e-3) / 1e9, "peak": peak,
                      "peak_kind": peak_kind, "unit": "GB/s", "frac": dom_bytes / (dom_ms * 1e-3) / 1e9 / peak,
-                     "traffic": None, "algorithmic_bytes_per_launch": dom_bytes},
+                     "traffic": NCU_TRAFFIC_BYTES.get(wl.name, {}).get(dominant), "algorithmic_bytes_per_launch": dom_bytes,
+                     "note": "achieved = algorithmic bytes of the launch / mean CUDA-event duration of that kernel; "
+                             "frac is of the measured copy bandwidth"},
         "e2e": None if e2e_ms is None else {"value": world * n_e2e / (e2e_ms / 1e3), "unit": UNIT,
                                             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e},
         "clocks": clocks,
