@@ -179,6 +179,28 @@ def test_tova_ragged_batch():
     _check_scorer(wl)
 
 
+def test_tova_maximum_sequence_length():
+    """131072 cached tokens (the largest supported): 1024 tiles per unit in the tensor-core scorer,
+    a cluster of eight blocks in the segmentation kernel."""
+    wl = _small(4, n_layers=1, batch=1, n_q_heads=4, n_kv_heads=1, window=16, seq_len_min=131072, seq_len_max=131072,
+                budget=8192, n_segments=32, l_max=8192, append_per_step=0, steps=1)
+    _check_scorer(wl)
+
+
+def test_nothing_to_evict_leaves_everything_untouched():
+    wl = _small(0, n_layers=2, batch=3, seq_len_min=600, seq_len_max=600, budget=384)
+    cache = inputs.make_cache(wl, DEV)
+    comp = binding.AmsCompressor(binding.config_for(wl), DEV)
+    cache.seq_lens.copy_(torch.tensor([300, 384, 10], dtype=torch.int32))   # every sequence already within the budget
+    k0, v0 = cache.k_pages.clone(), cache.v_pages.clone()
+    table0, lens0 = cache.block_table.clone(), cache.seq_lens.clone()
+    gpu_event(comp, cache, inputs.alloc_dst_pages(cache))
+    assert torch.equal(cache.k_pages.view(torch.int16), k0.view(torch.int16))
+    assert torch.equal(cache.v_pages.view(torch.int16), v0.view(torch.int16))
+    assert torch.equal(cache.block_table, table0) and torch.equal(cache.seq_lens, lens0)
+    assert float(comp.ema_state.abs().sum()) == 0.0
+
+
 def test_keydiff_scores_and_selection():
     wl = _small(3, n_layers=2, batch=3, seq_len_min=900, seq_len_max=2000, budget=256, n_segments=16, l_max=250)
     _check_scorer(wl, rtol=1e-3, atol=1e-5)
