@@ -354,7 +354,12 @@ __global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, i
 
     // ---- prefix of the mass at each segment end, written by the thread that owns the
     //      segment's last token; segment mass = difference of consecutive ends
+    bool owns_end = false; // most threads lie strictly inside one segment and have nothing to write
     if (valid) {
+        const int n_valid = __popc(valid);
+        owns_end = (newseg >> 1) != 0u || t_base + my0 + n_valid == bounds[seg0 + __popc(newseg) + 1];
+    }
+    if (owns_end) {
         int s = seg0;
         u64 run = exc;
 #pragma unroll
@@ -738,13 +743,24 @@ __global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, i
     } else {
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
-            const int t = t_base + my0 + i;
             if (kept_bits & (1u << i)) {
-                keep[pos] = t;
+                keep[pos] = t_base + my0 + i;
                 if (ema_on) credit[pos] = crs[i * nt + tid];
                 ++pos;
             }
-            if (ema_on && my0 + i < n_loc && t >= p.Tk) credit[t] = 0.0f;
+        }
+        if (ema_on) { // rows beyond the budget: whole groups of four with one store
+#pragma unroll
+            for (int q = 0; q < VPT / 4; ++q) {
+                const int t = t_base + my0 + 4 * q;
+                if (my0 + 4 * q + 3 < n_loc && t >= p.Tk) {
+                    *reinterpret_cast<float4 *>(credit + t) = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        if (my0 + 4 * q + k < n_loc && t + k >= p.Tk) credit[t + k] = 0.0f;
+                }
+            }
         }
     }
     if (cs > 1) cluster.sync(); // nobody leaves while a neighbour may still read its shared memory
