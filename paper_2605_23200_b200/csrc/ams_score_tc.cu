@@ -5,7 +5,8 @@
 // takes the contiguous tile range [c * tpc, (c + 1) * tpc).  Inside a block:
 //   warp 0      TMA producer: query block of the current unit, then one 32 KB K tile per
 //               stage (eight 16-token pages, one 4 KB copy each, 128-byte swizzle);
-//   warp 1      MMA issuer (one lane): per (tile, 128-row query block) eight
+//   warps 1, 3  MMA issuers (one lane each, one per consumer warpgroup, tiles in turn): per
+//               (tile, 128-row query block) eight
 //               tcgen05.mma m128 n128 k16 into one of four 128-column TMEM slots (two per
 //               consumer warpgroup, used in turn);
 //   warps 4-11  two consumer warpgroups, alternating tiles; thread i of a warpgroup owns
@@ -36,7 +37,7 @@ constexpr int kMaxStages = 6;
 
 struct TcShared {
     unsigned long long kfull[kMaxStages], kempty[kMaxStages], tfull[kSlots], tempty[kSlots];
-    unsigned long long qfull, qempty, done;
+    unsigned long long qfull, qempty, done[2];
     uint32_t tmem_base;
     int abort_flag;
     int tiles_lh, tpc;
@@ -108,8 +109,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
         for (int i = 0; i < kMaxStages; ++i) { mbar_init(smem_u32(&sh.kfull[i]), 1); mbar_init(smem_u32(&sh.kempty[i]), 1); }
         for (int i = 0; i < kSlots; ++i) { mbar_init(smem_u32(&sh.tfull[i]), 1); mbar_init(smem_u32(&sh.tempty[i]), 4); }
         mbar_init(smem_u32(&sh.qfull), 1);
-        mbar_init(smem_u32(&sh.qempty), 1);
-        mbar_init(smem_u32(&sh.done), 1);
+        mbar_init(smem_u32(&sh.qempty), 2); // both MMA issuers release the query block
+        mbar_init(smem_u32(&sh.done[0]), 1);
+        mbar_init(smem_u32(&sh.done[1]), 1);
         sh.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -179,23 +181,26 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
                         if (mbar_try_wait(smem_u32(&sh.kfull[k % NS]), (uint32_t)((k / NS) & 1))) break;
                 }
             }
-        } else if (warp == 1) {
-            // ------------------------------------------------------------ MMA issuer
+        } else if (warp == 1 || warp == 3) {
+            // ------------------------------------------------------------ MMA issuers
+            // One thread per consumer warpgroup, taking the tiles in turn: a tile costs its issuer a
+            // chain of long waits (two barriers, eight MMAs, two commits) that is longer than the
+            // tile's share of the HBM stream, so a single issuer would be the bottleneck.
             if (lane == 0) {
-                int kit = 0, seg = 0;
-                int wsit[2] = {0, 0}; // accumulator slots handed to each consumer warpgroup so far
+                const int wg = warp >> 1; // issuer 0 feeds warpgroup 0 (even tiles), issuer 1 warpgroup 1
+                int kit = 0, seg = 0, wsit = 0; // wsit: accumulator slots handed to the warpgroup so far
                 bool ok = true;
                 for (long long g = g_begin; g < g_end && ok;) {
                     const Segment s = decode_segment(p, prefix, tiles_lh, tpc, g, g_end, my_h);
                     ok = mbar_wait(smem_u32(&sh.qfull), (uint32_t)(seg & 1), abort_flag);
                     for (int i = 0; i < s.n && ok; ++i, ++kit) {
+                        if ((kit & 1) != wg) continue;
                         const int st = kit % NS;
                         ok = mbar_wait(smem_u32(&sh.kfull[st]), (uint32_t)((kit / NS) & 1), abort_flag);
-                        const int wg = kit & 1;
-                        for (int rb = 0; rb < n_rb && ok; ++rb, ++wsit[wg]) {
+                        for (int rb = 0; rb < n_rb && ok; ++rb, ++wsit) {
                             // warpgroup wg owns slots 2 wg and 2 wg + 1, used in turn
-                            const int slot = 2 * wg + (wsit[wg] & 1);
-                            ok = mbar_wait(smem_u32(&sh.tempty[slot]), (uint32_t)(((wsit[wg] >> 1) & 1) ^ 1), abort_flag);
+                            const int slot = 2 * wg + (wsit & 1);
+                            ok = mbar_wait(smem_u32(&sh.tempty[slot]), (uint32_t)(((wsit >> 1) & 1) ^ 1), abort_flag);
                             if (!ok) break;
                             tc_fence_after();
                             const uint32_t qa = smem_u32(Qs + (size_t)rb * kTileBytes), ka = smem_u32(Ks + (size_t)st * kTileBytes);
@@ -215,9 +220,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
                     ++seg;
                 }
                 // all tensor work issued by this thread has finished before TMEM is released
-                tc_commit(smem_u32(&sh.done));
+                tc_commit(smem_u32(&sh.done[wg]));
                 for (uint32_t i = 0; i < kWaitLimit; ++i)
-                    if (mbar_try_wait(smem_u32(&sh.done), 0)) break;
+                    if (mbar_try_wait(smem_u32(&sh.done[wg]), 0)) break;
             }
             __syncwarp();
         } else if (warp >= 4) {
