@@ -229,7 +229,7 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
     p.slice_len = y.slice_len; p.n_slices = y.n_slices;
     p.rows_pad = scorer_id == AMS_SCORER_TOVA ? rows_padded(p.rows) : kHeadDim;
     p.tc_tpc_min = tc_tiles_per_block_min(y.T_cap);
-    p.tc_stages = p.rows_pad <= 128 ? 4 : (p.rows_pad <= 256 ? 3 : 2);
+    p.tc_stages = p.rows_pad <= 256 ? 4 : 2; // even: each stage then belongs to one of the two MMA issuers
     p.status = (int *)(st->ws + y.status);
     p.fcnt = (int *)(st->ws + y.ctrl);
     p.fflag = p.fcnt + (size_t)c.n_layers * c.max_batch * c.n_kv_heads;

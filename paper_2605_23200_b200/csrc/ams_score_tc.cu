@@ -417,6 +417,9 @@ size_t tova_tc_smem_bytes(const DevParams &p)
 
 int launch_score_tova_tc(const DevParams &p, LaunchCtx &ctx)
 {
+    // With two MMA issuers taking tiles in turn, an even ring depth gives every stage to one issuer, which
+    // then sees all phases of the stage's barrier in order (a parity wait must not skip a phase).
+    if (p.tc_stages < 2 || (p.tc_stages & 1)) return AMS_ERR_UNSUPPORTED;
     EncodeTiledFn enc = encode_fn();
     if (!enc) return AMS_ERR_CUDA;
     CUtensorMap k_map, q_map;
