@@ -40,6 +40,7 @@ struct TcShared {
     unsigned long long qfull, qempty, done[2];
     uint32_t tmem_base;
     int abort_flag;
+    float wmax[2][8];
     int tiles_lh, tpc;
     long long n_tiles;
 };
@@ -237,7 +238,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
                 const int T = s.T;
                 float m[4], z[4];
                 int lastv[4];
-                const float *fin = p.fin + (size_t)s.uid * (p.rows_pad + 8);
                 float *fs = fin_s + (seg & 1) * p.rows_pad;
                 float pmax = 0.0f;
                 if (PHASE == 1) {
@@ -248,9 +248,28 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
                         lastv[rb] = r < p.rows ? (p.causal ? T - p.W + (r % p.W) : T - 1) : -1;
                     }
                 } else {
-                    for (int r = (warp - 4) * 32 + lane; r < p.rows_pad; r += 256) fs[r] = fin[r];
-                    pmax = fin[p.rows_pad];
+                    // merge the statistics the blocks of the first pass left for this unit, in block
+                    // order: b_r = M_r + log2 Z_r per row, and the window maximum 1 / min_r Z_r
+                    const int nt_u = prefix[s.b + 1] - prefix[s.b];
+                    const long long ustart = g - s.tile0;
+                    const int n_parts = (int)((ustart + nt_u - 1) / tpc) - (int)(ustart / tpc) + 1;
+                    float best = 0.0f;
+                    for (int r = (warp - 4) * 32 + lane; r < p.rows_pad; r += 256) {
+                        float mm = -INFINITY, zz = 0.0f;
+                        for (int q = 0; q < n_parts; ++q) {
+                            const float2 v = __ldcg(reinterpret_cast<const float2 *>(p.part) + ((size_t)s.uid * p.n_slices + q) * p.rows_pad + r);
+                            lse_merge(mm, zz, v.x, v.y);
+                        }
+                        const bool live = r < p.rows && zz > 0.0f;
+                        fs[r] = live ? mm + log2f(zz) : INFINITY; // padding rows contribute nothing
+                        if (live) best = fmaxf(best, 1.0f / zz);
+                    }
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, o));
+                    if (lane == 0) sh.wmax[seg & 1][warp - 4] = best;
                     asm volatile("bar.sync 1, 256;" ::: "memory");
+#pragma unroll
+                    for (int w = 0; w < 8; ++w) pmax = fmaxf(pmax, sh.wmax[seg & 1][w]);
                 }
                 for (int i = 0; i < s.n && ok; ++i, ++kit) {
                     if ((kit & 1) != wg) continue;
@@ -372,39 +391,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
 }
 
-// Per unit: merge the parts written by the blocks that shared the unit, in block order.
-__global__ void __launch_bounds__(128) k_tova_combine_tc(DevParams p, int tc_grid)
-{
-    __shared__ u64 scratch[40];
-    __shared__ int prefix[1025];
-    __shared__ int s_tiles_lh, s_tpc;
-    __shared__ long long s_n;
-    tc_partition(p, tc_grid, prefix, &s_tiles_lh, &s_n, &s_tpc);
-    const int uid = blockIdx.x;
-    const int b = (uid / p.H) % p.B, l = uid / (p.H * p.B);
-    const int nt = prefix[b + 1] - prefix[b];
-    if (nt == 0) return;
-    const long long ustart = (long long)l * s_tiles_lh + prefix[b];
-    const int n_parts = (int)((ustart + nt - 1) / s_tpc) - (int)(ustart / s_tpc) + 1;
-    float *fin = p.fin + (size_t)uid * (p.rows_pad + 8);
-    float best = 0.0f;
-    for (int r = threadIdx.x; r < p.rows_pad; r += blockDim.x) {
-        float m = -INFINITY, z = 0.0f;
-        for (int s = 0; s < n_parts; ++s) {
-            const float2 v = reinterpret_cast<const float2 *>(p.part)[((size_t)uid * p.n_slices + s) * p.rows_pad + r];
-            lse_merge(m, z, v.x, v.y);
-        }
-        if (r < p.rows && z > 0.0f) {
-            fin[r] = m + log2f(z);
-            best = fmaxf(best, 1.0f / z);
-        } else {
-            fin[r] = INFINITY;
-        }
-    }
-    best = block_max_f32(best, scratch);
-    if (threadIdx.x == 0) fin[p.rows_pad] = best;
-}
-
 } // namespace
 
 bool tova_tc_supported(const DevParams &p) { return p.rows >= 64 && p.rows_pad % 128 == 0 && p.rows_pad <= 512 && p.B <= 1024 && p.H <= 64; }
@@ -467,8 +453,6 @@ int launch_score_tova_tc(const DevParams &p, LaunchCtx &ctx)
     const int grid = groups * p.H;
     k_tova_tc<1><<<grid, kTcThreads, smem, ctx.s>>>(p, k_map, q_map);
     ctx.mark(kKernScore1);
-    k_tova_combine_tc<<<p.L * p.B * p.H, 128, 0, ctx.s>>>(p, groups);
-    ctx.mark(kKernScoreCombine);
     k_tova_tc<2><<<grid, kTcThreads, smem, ctx.s>>>(p, k_map, q_map);
     ctx.mark(kKernScore2);
     return cudaGetLastError() == cudaSuccess ? AMS_OK : AMS_ERR_CUDA;
