@@ -37,6 +37,11 @@
  * Decisions (cut positions, quotas, kept indices) are taken in integer arithmetic
  * on fixed-point images of the mass, so they do not depend on summation order.
  *
+ * Scorer selection is automatic (query rows per KV head >= 64: tensor-core path, otherwise the
+ * mma.sync path).  Setting the environment variable AMS_FUSED_SCORER=1 selects an experimental
+ * scorer that reads K once (query rows padded to 128, sequences up to 148 tiles of 128 tokens);
+ * it is slower than the default at the sizes measured so far.
+ *
  * Errors: every function returns AMS_OK (0) or a negative code.  Calls are
  * asynchronous on `stream`; conditions found on the device (a sequence longer
  * than max_seq_len, a window longer than a sequence, a bounded wait that ran out)
