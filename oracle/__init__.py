@@ -126,6 +126,18 @@ def score_keydiff(k_pages, layer, h, table_row, T):
 
 # --------------------------------------------------------------------------- stages
 
+def smooth_usage(u, k):
+    """Zero-padded 1-D average pooling of the usage scores, window k (odd), stride 1
+    (Algorithm 1 step 1, optional smoothing)."""
+    u = _f32(u)
+    if k < 1 or k % 2 == 0:
+        raise ValueError("pool kernel must be odd and >= 1")
+    out = np.empty_like(u)
+    lib().orc_smooth_usage(_p(u, ctypes.c_float), ctypes.c_int32(u.shape[0]), ctypes.c_int32(k),
+                           _p(out, ctypes.c_float))
+    return out
+
+
 def mass(u, eps):
     """Eq. 1 on fixed-point weights.  Returns (A uint64[T], SA, m float32[T])."""
     u = _f32(u)
@@ -267,7 +279,7 @@ SCORER_TOVA, SCORER_KEYDIFF, SCORER_EXTERNAL = 0, 1, 2
 
 def compress(k_pages, v_pages, block_table, seq_lens, obs_queries, credit, budget, prm: Params,
              scorer_id, dst_pages, *, n_q_heads=None, causal=True, ext_scores=None, units=None,
-             do_gather=True, threads=1):
+             do_gather=True, threads=1, pool_kernel=1, decoupled=False, ext_usage=None):
     """One compression event over every layer, sequence and KV head.
 
     k_pages / v_pages: uint16 [L][P][page][H][D] (modified: kept rows are written into
@@ -275,7 +287,13 @@ def compress(k_pages, v_pages, block_table, seq_lens, obs_queries, credit, budge
     (rewritten as the event leaves them); obs_queries uint16 [L][B][Hq][W][D] or None;
     credit float32 [L][B][H][T_cap] (updated in place); ext_scores float32 like credit for
     SCORER_EXTERNAL.  `units`: optional subset of (layer, b, h) to compute (for sampling);
-    the table update is skipped then.  Returns {(layer,b,h): UnitResult} with `.scores`."""
+    the table update is skipped then.
+
+    Mass signal: by default the usage u that defines the mass is the scorer's score g.
+    `decoupled` (SCORER_KEYDIFF with observation queries): u = window attention, g = key-only
+    score.  `ext_usage` (SCORER_EXTERNAL): u given separately from g.  `pool_kernel` > 1
+    smooths u (never g) before Eq. 1.  Returns {(layer,b,h): UnitResult} with `.scores` (g)
+    and `.usage` (u after smoothing)."""
     L, P, page, H, D = k_pages.shape
     B = seq_lens.shape[0]
     T_cap = credit.shape[-1]
@@ -286,15 +304,25 @@ def compress(k_pages, v_pages, block_table, seq_lens, obs_queries, credit, budge
     def one(unit):
         l, b, h = unit
         T = int(seq_lens[b])
+        u = None
         if scorer_id == SCORER_TOVA:
             W = obs_queries.shape[3]
             s = score_tova(k_pages, l, h, block_table[b], T, obs_queries[l, b, h * G:(h + 1) * G], G, W, causal)
         elif scorer_id == SCORER_KEYDIFF:
             s = score_keydiff(k_pages, l, h, block_table[b], T)
+            if decoupled:
+                W = obs_queries.shape[3]
+                u = score_tova(k_pages, l, h, block_table[b], T, obs_queries[l, b, h * G:(h + 1) * G], G, W, causal)
         else:
             s = _f32(ext_scores[l, b, h, :T])
-        res = select_unit(s, None, credit[l, b, h, :T], budget, prm)
+            if ext_usage is not None:
+                u = _f32(ext_usage[l, b, h, :T])
+        u = s if u is None else u
+        if pool_kernel > 1:
+            u = smooth_usage(u, pool_kernel)
+        res = select_unit(u, s, credit[l, b, h, :T], budget, prm)
         res.scores = s
+        res.usage = u
         return unit, res
 
     if threads > 1:

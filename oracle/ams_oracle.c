@@ -24,7 +24,8 @@
  * exact rational brute force; uniform mass => equal segments; quotas summing to
  * the budget with their bounds; one segment => library top-k; beta = 1 => EMA
  * off; lambda = 0 => credit equals mass; gather equals dense indexing; TOVA
- * with one query row => library softmax; KeyDiff => library cosine similarity.
+ * with one query row => library softmax; KeyDiff => library cosine similarity;
+ * usage smoothing => library zero-padded average pooling and a hand-computed case.
  * Parity unpinned (invariants only): merge direction and the order of merge vs
  * split; the choice of "roughly equal" split sizes; rounding rule of the quota
  * share; the padding value of the causal observation window when W > 1.
@@ -190,6 +191,25 @@ void orc_fixed_point(const float *x, int32_t T, uint64_t *A, uint64_t *sum_out)
         for (int t = 0; t < T; ++t) A[t] = 0;
     }
     *sum_out = s;
+}
+
+/* Optional smoothing of the usage scores along the sequence before Eq. 1 (Algorithm 1,
+ * step 1: "optionally smooth"; the default configuration of the implementation-details
+ * appendix names a small 1-D average pooling).  Window of k positions (k odd) centred on
+ * t, positions outside [0, T) count as zero and the divisor is always k (the convention
+ * of a zero-padded average pooling with stride 1).  The sum runs over the positions inside
+ * the sequence from left to right in fp32, one rounding per addition, then one division:
+ * a fixed order, so that the result has one value.  k = 1 leaves u as it is. */
+void orc_smooth_usage(const float *u, int32_t T, int32_t k, float *out)
+{
+    const int r = k / 2;
+    for (int t = 0; t < T; ++t) {
+        if (k <= 1) { out[t] = u[t]; continue; }
+        float s = 0.0f;
+        const int lo = t - r < 0 ? 0 : t - r, hi = t + r > T - 1 ? T - 1 : t + r;
+        for (int j = lo; j <= hi; ++j) s = s + u[j];
+        out[t] = s / (float)k;
+    }
 }
 
 void orc_weights(const float *u, int32_t T, float eps, float *w)

@@ -459,3 +459,82 @@ def test_keydiff_is_negative_cosine_to_mean_key():
     mu = x[0, 0, :, 0].double().mean(0)
     assert abs(g[3] + float(7.0 * mu[5] / (7.0 * mu.norm()))) < 1e-6
     assert g[4] > 0.9 and g[0] < -0.9
+
+
+# ----------------------------------------------------------------------------- usage smoothing, decoupled signals
+
+def test_usage_smoothing_hand_computed_and_library_pooling():
+    # small integers: every partial sum and quotient by 4-bit-exact divisors is exact
+    u = np.array([4, 8, 0, 12, 16, 4], np.float32)
+    assert oracle.smooth_usage(u, 1).tolist() == u.tolist()
+    assert oracle.smooth_usage(u, 3).tolist() == [np.float32(x) / np.float32(3) for x in (12, 12, 20, 28, 32, 20)]
+    want5 = [np.float32(x) / np.float32(5) for x in (12, 24, 40, 40, 32, 32)]
+    assert oracle.smooth_usage(u, 5).tolist() == want5
+    # a window wider than the sequence still divides by k
+    assert oracle.smooth_usage(np.array([3, 6], np.float32), 7).tolist() == [np.float32(9) / np.float32(7)] * 2
+    # against a library's zero-padded average pooling (stride 1, padding k // 2)
+    rng = np.random.default_rng(5)
+    x = np.exp(rng.standard_normal(1000)).astype(np.float32)
+    for k in (3, 5, 7, 9):
+        ref = torch.nn.functional.avg_pool1d(torch.from_numpy(x).double()[None, None], k, stride=1, padding=k // 2)[0, 0]
+        np.testing.assert_allclose(oracle.smooth_usage(x, k), ref.numpy(), rtol=2e-6)
+    with pytest.raises(ValueError):
+        oracle.smooth_usage(x, 4)
+
+
+def _event_inputs(rng, T=300, W=4, Hq=4, H=2):
+    pages, table, dense = _tiny_cache(rng, T=T, P=T // 16 + 12)
+    q = torch.randn((1, 1, Hq, W, 128)).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    dst = np.arange(T // 16 + 2, T // 16 + 2 + 4, dtype=np.int32)[None]
+    return pages, table, q, dst
+
+
+def test_smoothing_changes_the_mass_only_and_decoupled_signals_split_roles():
+    """Smoothing and a separate usage signal act on the mass (hence on segments and quotas);
+    inside a segment tokens are still ranked by the base score g."""
+    rng = np.random.default_rng(31)
+    torch.manual_seed(31)
+    T, Tk = 300, 64
+    pages, table, q, dst = _event_inputs(rng, T=T)
+    prm = Params(n_segments=6, l_min=8, l_max=0, q_min=1, n_sink=2, n_last=4, ema_lambda=0.9, ema_beta=1.0, eps=1e-8)
+    lens = np.array([T], np.int32)
+    tab = table[None].copy()
+    credit = np.zeros((1, 1, 2, T), np.float32)
+
+    def run(**kw):
+        return oracle.compress(pages.copy(), pages.copy(), tab.copy(), lens.copy(), q, credit.copy(), Tk, prm,
+                               kw.pop("scorer", oracle.SCORER_TOVA), dst, n_q_heads=4, do_gather=False, **kw)
+
+    base = run()
+    pooled = run(pool_kernel=5)
+    for unit in base:
+        g = base[unit].scores
+        assert (pooled[unit].scores == g).all()                                  # g is not smoothed
+        assert (pooled[unit].usage == oracle.smooth_usage(g, 5)).all()
+        _, _, m = oracle.mass(oracle.smooth_usage(g, 5), prm.eps)
+        assert (pooled[unit].mass == m).all()
+        # selection inside each segment of the pooled run is the top-q of g there
+        r = pooled[unit]
+        for i in range(r.n_seg):
+            a, b = r.bounds[i], r.bounds[i + 1]
+            order = sorted(range(a, b), key=lambda t: (-g[t], t))[: r.quotas[i]]
+            assert set(order) <= set(r.keep_idx.tolist())
+    # decoupled: mass from the window attention, ranking from the key-only score
+    dec = run(scorer=oracle.SCORER_KEYDIFF, decoupled=True)
+    kd = run(scorer=oracle.SCORER_KEYDIFF)
+    for unit in base:
+        assert (dec[unit].usage == base[unit].scores).all() and (dec[unit].scores == kd[unit].scores).all()
+        assert (dec[unit].bounds == base[unit].bounds).all() and (dec[unit].quotas == base[unit].quotas).all()
+        r, g = dec[unit], kd[unit].scores
+        for i in range(r.n_seg):
+            a, b = r.bounds[i], r.bounds[i + 1]
+            order = sorted(range(a, b), key=lambda t: (-g[t], t))[: r.quotas[i]]
+            assert set(order) <= set(r.keep_idx.tolist())
+    # an external usage signal plays the same role
+    ext_g = rng.standard_normal((1, 1, 2, T)).astype(np.float32)
+    ext_u = np.exp(rng.standard_normal((1, 1, 2, T))).astype(np.float32)
+    both = run(scorer=oracle.SCORER_EXTERNAL, ext_scores=ext_g, ext_usage=ext_u)
+    only_u = run(scorer=oracle.SCORER_EXTERNAL, ext_scores=ext_u)
+    for unit in both:
+        assert (both[unit].bounds == only_u[unit].bounds).all() and (both[unit].quotas == only_u[unit].quotas).all()
+        assert (both[unit].mass == only_u[unit].mass).all()
