@@ -87,13 +87,20 @@ typedef struct {
     float ema_beta;                          /* weight of the current mass; 1 = credit unused */
     float eps;                               /* Eq. 1 epsilon, > 0                            */
     int32_t causal_window;                   /* 1: window query j sees tokens <= T - W + j    */
+    int32_t pool_kernel;                     /* odd, 1..63: width of the average pooling applied
+                                                to the usage scores before Eq. 1 (Algorithm 1
+                                                step 1, optional smoothing); 1 = none         */
+    int32_t decoupled;                       /* 1: reserve room for a mass signal that differs
+                                                from the base scores (see ams_compress)       */
 } ams_config;
 
 /* Optional device outputs for inspection and tests; any member may be NULL.
  * T = max_seq_len, C = ams_segment_capacity(cfg).  Units that were skipped
  * (seq_len <= budget) are left untouched. */
 typedef struct {
-    float *scores;       /* [L][batch][H][T]   base scores g (= usage u)                    */
+    float *scores;       /* [L][batch][H][T]   base scores g                                */
+    float *usage;        /* [L][batch][H][T]   usage u the mass is built from (after smoothing;
+                                               equals g unless smoothed or decoupled)       */
     float *mass;         /* [L][batch][H][T]   Eq. 1 mass of the current event              */
     int32_t *n_segments; /* [L][batch][H]      segments after merge and split               */
     int32_t *seg_bounds; /* [L][batch][H][C+1] boundaries a_0 = 0 < ... < a_n = seq_len     */
@@ -102,8 +109,8 @@ typedef struct {
 } ams_debug_views;
 
 /* Paper defaults: segment mass 0.1 (n_segments = 10 is passed per call), lengths
- * 16 / 256, q_min 1, lambda = beta = 0.9, 4 sinks; n_last 16, eps 1e-8.  Geometry
- * and capacities are zeroed and must be filled by the caller. */
+ * 16 / 256, q_min 1, lambda = beta = 0.9, 4 sinks; n_last 16, eps 1e-8; pool_kernel 1 (no
+ * smoothing), decoupled 0.  Geometry and capacities are zeroed and must be filled by the caller. */
 void ams_config_default(ams_config *cfg);
 
 /* Sizes of the caller-allocated device buffers; 0 if the configuration is invalid. */
@@ -128,15 +135,24 @@ int ams_init_state(const ams_config *cfg, void *ema_state, void *workspace, size
  *  obs_queries, window : may be NULL / 0 for AMS_SCORER_KEYDIFF and AMS_SCORER_EXTERNAL.
  *  ema_state        : the buffer given to ams_init_state (or a restored copy of it).
  *  n_segments       : S, the number of mass quantiles (segment mass 1/S), 1..max_segments.
- *  ext_scores       : AMS_SCORER_EXTERNAL only: fp32 [L][batch][H][max_seq_len] (16-byte aligned) scores used both
- *                     as usage and as base scores.
+ *  ext_scores       : AMS_SCORER_EXTERNAL only: fp32 [L][batch][H][max_seq_len] (16-byte aligned) base
+ *                     scores g; also the usage u unless ext_usage is given.
+ *  ext_usage        : AMS_SCORER_EXTERNAL only, optional (NULL: u = g): fp32, same shape and alignment,
+ *                     the usage u.
+ * Mass signal (Algorithm 1 step 1; the runtime section's "decoupled mass and selection scores"):
+ * the mass is built from the usage u, tokens inside a segment are ranked by the base score g.
+ * By default u = g = the scorer's output.  With cfg.decoupled = 1, AMS_SCORER_KEYDIFF and
+ * observation queries given (obs_queries != NULL, window >= 1), u is the window attention of
+ * AMS_SCORER_TOVA and g the key-only score.  cfg.pool_kernel = k > 1 replaces u (never g) by its
+ * zero-padded average over k neighbouring positions: u'_t = (sum of u_j, |j - t| <= k/2, j inside
+ * the sequence, added left to right in fp32) / k.
  *  dbg              : optional views, or NULL.
  * Calls on the same handle share the workspace and must not overlap on the GPU. */
 int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages, int32_t *block_table,
                  int32_t block_table_stride, int32_t *seq_lens, int32_t batch, const void *obs_queries,
                  int32_t window, void *ema_state, int32_t budget, int32_t n_segments, int32_t scorer_id,
-                 const int32_t *dst_pages, const float *ext_scores, const ams_debug_views *dbg,
-                 void *stream);
+                 const int32_t *dst_pages, const float *ext_scores, const float *ext_usage,
+                 const ams_debug_views *dbg, void *stream);
 
 /* Synchronises `stream`, then returns and clears the device status: AMS_OK or the
  * first device-side error.  detail[0..3] (host, may be NULL) receive the code, the
@@ -151,7 +167,7 @@ int32_t ams_last_launch_count(const ams_state *st);
  * device memory is allocated).  ams_get_kernel_times waits for the last call's final
  * event and writes AMS_KERNEL_SLOTS durations in milliseconds, one per kernel slot
  * named by ams_kernel_name (a slot launched more than once holds the sum). */
-#define AMS_KERNEL_SLOTS 6
+#define AMS_KERNEL_SLOTS 7
 int ams_set_profiling(ams_state *st, int enable);
 int ams_get_kernel_times(ams_state *st, float *ms);
 const char *ams_kernel_name(int32_t idx);

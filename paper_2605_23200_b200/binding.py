@@ -25,7 +25,7 @@ AMS_SCORER_TOVA, AMS_SCORER_KEYDIFF, AMS_SCORER_EXTERNAL = 0, 1, 2
 EXPORTS = ["ams_config_default", "ams_ema_state_bytes", "ams_workspace_bytes", "ams_segment_capacity",
            "ams_init_state", "ams_compress", "ams_get_status", "ams_last_launch_count", "ams_free",
            "ams_strerror", "ams_set_profiling", "ams_get_kernel_times", "ams_kernel_name", "ams_select_static"]
-KERNEL_SLOTS = 6
+KERNEL_SLOTS = 7
 
 
 class AmsConfig(ctypes.Structure):
@@ -33,11 +33,11 @@ class AmsConfig(ctypes.Structure):
                 ("n_layers", "n_q_heads", "n_kv_heads", "head_dim", "page_size", "max_batch", "max_seq_len",
                  "max_window", "max_budget", "max_segments", "l_min", "l_max", "q_min", "n_sink", "n_last")] + \
                [("ema_lambda", ctypes.c_float), ("ema_beta", ctypes.c_float), ("eps", ctypes.c_float),
-                ("causal_window", ctypes.c_int32)]
+                ("causal_window", ctypes.c_int32), ("pool_kernel", ctypes.c_int32), ("decoupled", ctypes.c_int32)]
 
 
 class AmsDebugViews(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_void_p) for n in ("scores", "mass", "n_segments", "seg_bounds", "quotas", "keep_idx")]
+    _fields_ = [(n, ctypes.c_void_p) for n in ("scores", "usage", "mass", "n_segments", "seg_bounds", "quotas", "keep_idx")]
 
 
 _lib = None
@@ -63,7 +63,7 @@ def lib() -> ctypes.CDLL:
         L.ams_compress.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
                                    ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_int32,
                                    ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_int32,
-                                   ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
+                                   ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                    ctypes.POINTER(AmsDebugViews), ctypes.c_void_p]
         L.ams_compress.restype = ctypes.c_int
         L.ams_get_status.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32)]
@@ -117,6 +117,7 @@ def _ptr(t):
 class DebugViews:
     """Device tensors that receive the library's intermediate results."""
     scores: torch.Tensor
+    usage: torch.Tensor
     mass: torch.Tensor
     n_segments: torch.Tensor
     seg_bounds: torch.Tensor
@@ -125,7 +126,8 @@ class DebugViews:
 
     def c(self) -> AmsDebugViews:
         return AmsDebugViews(*(t.data_ptr() for t in
-                               (self.scores, self.mass, self.n_segments, self.seg_bounds, self.quotas, self.keep_idx)))
+                               (self.scores, self.usage, self.mass, self.n_segments, self.seg_bounds, self.quotas,
+                                self.keep_idx)))
 
 
 class AmsCompressor:
@@ -159,13 +161,14 @@ class AmsCompressor:
         U = (c.n_layers, batch, c.n_kv_heads)
         return DebugViews(torch.zeros(U + (c.max_seq_len,), dtype=torch.float32, device=dev),
                           torch.zeros(U + (c.max_seq_len,), dtype=torch.float32, device=dev),
+                          torch.zeros(U + (c.max_seq_len,), dtype=torch.float32, device=dev),
                           torch.zeros(U, dtype=torch.int32, device=dev),
                           torch.zeros(U + (self.seg_cap + 1,), dtype=torch.int32, device=dev),
                           torch.zeros(U + (self.seg_cap,), dtype=torch.int32, device=dev),
                           torch.zeros(U + (budget,), dtype=torch.int32, device=dev))
 
     def compress(self, k_pages, v_pages, block_table, seq_lens, obs_queries, budget, n_segments, scorer_id,
-                 dst_pages, *, ext_scores=None, dbg: DebugViews | None = None, ema_state=None,
+                 dst_pages, *, ext_scores=None, ext_usage=None, dbg: DebugViews | None = None, ema_state=None,
                  stream: torch.cuda.Stream | None = None) -> None:
         """Enqueues one compression event on `stream` (default: torch's current stream)."""
         assert k_pages.is_contiguous() and v_pages.is_contiguous() and block_table.is_contiguous()
@@ -178,6 +181,7 @@ class AmsCompressor:
         rc = lib().ams_compress(self._h, _ptr(k_pages), _ptr(v_pages), k_pages.shape[1], _ptr(block_table),
                                 block_table.shape[1], _ptr(seq_lens), seq_lens.shape[0], _ptr(obs_queries), window,
                                 _ptr(ema), budget, n_segments, scorer_id, _ptr(dst_pages), _ptr(ext_scores),
+                                _ptr(ext_usage),
                                 ctypes.byref(views) if views is not None else None, ctypes.c_void_p(s.cuda_stream))
         if rc != AMS_OK:
             raise AmsError(rc, "ams_compress")
@@ -240,4 +244,5 @@ def config_for(wl, **kw) -> AmsConfig:
                           max_batch=wl.batch, max_seq_len=wl.max_seq_len, max_window=max(wl.window, 0),
                           max_budget=wl.budget, max_segments=max(wl.n_segments, 1), l_min=wl.l_min, l_max=wl.l_max,
                           q_min=wl.q_min, n_sink=wl.n_sink, n_last=wl.n_last, ema_lambda=wl.ema_lambda,
-                          ema_beta=wl.ema_beta, eps=wl.eps, **kw)
+                          ema_beta=wl.ema_beta, eps=wl.eps, pool_kernel=wl.pool_kernel, decoupled=int(wl.decoupled),
+                          **kw)

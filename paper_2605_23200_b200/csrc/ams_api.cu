@@ -8,7 +8,7 @@
 namespace ams {
 
 struct Layout {
-    size_t status, scores, cbuf, flags, n_seg, seg_bounds, quotas, keep_idx, part, fin, ctrl, finz, total;
+    size_t status, scores, usage, cbuf, flags, n_seg, seg_bounds, quotas, keep_idx, part, fin, ctrl, finz, total;
     int units, T_cap, seg_cap, n_slices, slice_len, rows_pad_cap;
 };
 
@@ -26,6 +26,8 @@ static bool config_ok(const ams_config *c, int *why)
     if (!(c->ema_lambda >= 0.0f && c->ema_lambda < 1.0f)) return false;
     if (!(c->ema_beta >= 0.0f && c->ema_beta <= 1.0f)) return false;
     if (!(c->eps > 0.0f) || !(c->eps < 1e30f)) return false;
+    if (c->pool_kernel < 1 || c->pool_kernel > 63 || !(c->pool_kernel & 1)) return false;
+    if (c->decoupled != 0 && c->decoupled != 1) return false;
     *why = AMS_ERR_UNSUPPORTED;
     if (c->head_dim != kHeadDim || c->page_size != kPage) return false;
     if (c->n_q_heads % c->n_kv_heads) return false;
@@ -84,6 +86,8 @@ static Layout make_layout(const ams_config *c)
     size_t off = 0;
     y.status = off;     off = align_up(off + 64, 256);
     y.scores = off;     off = align_up(off + U * T * 4, 256);
+    // second per-token array: the usage when it is smoothed or comes from another scorer than the base scores
+    y.usage = off;      off = align_up(off + ((c->pool_kernel > 1 || c->decoupled) ? U * T * 4 : 0), 256);
     y.cbuf = off;       off = align_up(off + U * T * 8, 256);
     y.flags = off;      off = align_up(off + U * T, 256);
     y.n_seg = off;      off = align_up(off + U * 4, 256);
@@ -134,6 +138,8 @@ void ams_config_default(ams_config *cfg)
     cfg->ema_beta = 0.9f;
     cfg->eps = 1e-8f;
     cfg->causal_window = 1;
+    cfg->pool_kernel = 1;
+    cfg->decoupled = 0;
 }
 
 size_t ams_ema_state_bytes(const ams_config *cfg)
@@ -187,7 +193,8 @@ int ams_init_state(const ams_config *cfg, void *ema_state, void *workspace, size
 int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages, int32_t *block_table,
                  int32_t block_table_stride, int32_t *seq_lens, int32_t batch, const void *obs_queries,
                  int32_t window, void *ema_state, int32_t budget, int32_t n_segments, int32_t scorer_id,
-                 const int32_t *dst_pages, const float *ext_scores, const ams_debug_views *dbg, void *stream)
+                 const int32_t *dst_pages, const float *ext_scores, const float *ext_usage, const ams_debug_views *dbg,
+                 void *stream)
 {
     if (!st || !k_pages || !v_pages || !block_table || !seq_lens || !ema_state || !dst_pages) return AMS_ERR_INVALID_ARG;
     const ams_config &c = st->cfg;
@@ -202,7 +209,12 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
     } else if (scorer_id != AMS_SCORER_KEYDIFF) {
         return AMS_ERR_INVALID_ARG;
     }
-    if (((uintptr_t)k_pages | (uintptr_t)v_pages | (uintptr_t)obs_queries | (uintptr_t)ema_state | (uintptr_t)ext_scores) & 15) return AMS_ERR_INVALID_ARG;
+    if (ext_usage && scorer_id != AMS_SCORER_EXTERNAL) return AMS_ERR_INVALID_ARG;
+    // key-only base scores with the window attention as mass signal
+    const bool split = scorer_id == AMS_SCORER_KEYDIFF && c.decoupled && obs_queries && window >= 1;
+    if (split && window > c.max_window) return AMS_ERR_INVALID_ARG;
+    if (((uintptr_t)k_pages | (uintptr_t)v_pages | (uintptr_t)obs_queries | (uintptr_t)ema_state | (uintptr_t)ext_scores |
+         (uintptr_t)ext_usage) & 15) return AMS_ERR_INVALID_ARG;
 
     const Layout &y = st->lay;
     cudaStream_t s = (cudaStream_t)stream;
@@ -219,8 +231,12 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
     p.block_table = block_table; p.bt_stride = block_table_stride; p.seq_lens = seq_lens;
     p.q = (const __nv_bfloat16 *)obs_queries; p.ema = (float *)ema_state; p.dst_pages = dst_pages;
     p.scores = (float *)(st->ws + y.scores);
-    p.usage = scorer_id == AMS_SCORER_EXTERNAL ? ext_scores : p.scores;
-    if (scorer_id == AMS_SCORER_EXTERNAL) p.scores = const_cast<float *>(ext_scores);
+    p.usage = p.scores;
+    if (scorer_id == AMS_SCORER_EXTERNAL) {
+        p.scores = const_cast<float *>(ext_scores);
+        p.usage = ext_usage ? ext_usage : ext_scores;
+    }
+    float *usage_buf = (float *)(st->ws + y.usage);
     p.cbuf = (u64 *)(st->ws + y.cbuf); p.flags = st->ws + y.flags;
     p.n_seg = (int *)(st->ws + y.n_seg); p.seg_bounds = (int *)(st->ws + y.seg_bounds);
     p.quotas = (int *)(st->ws + y.quotas); p.keep_idx = (int *)(st->ws + y.keep_idx);
@@ -241,14 +257,34 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
     ctx.ev = st->profiling ? st->ev : nullptr;
     ctx.max_ev = 32;
     ctx.begin();
-    if (scorer_id == AMS_SCORER_TOVA) rc = launch_score_tova(p, ctx);
-    else if (scorer_id == AMS_SCORER_KEYDIFF) rc = launch_score_keydiff(p, ctx);
+    if (scorer_id == AMS_SCORER_TOVA) {
+        rc = launch_score_tova(p, ctx);
+    } else if (scorer_id == AMS_SCORER_KEYDIFF) {
+        if (split) {
+            // the window attention goes through the score array into the usage array (smoothed on the way
+            // if asked for); the key-only score then takes the score array
+            DevParams pt = p;
+            pt.W = window;
+            pt.rows = pt.G * window;
+            pt.rows_pad = rows_padded(pt.rows);
+            pt.tc_stages = pt.rows_pad <= 256 ? 4 : 2;
+            rc = launch_score_tova(pt, ctx);
+            if (rc == AMS_OK) rc = launch_smooth_usage(p, p.scores, usage_buf, c.pool_kernel, ctx);
+            p.usage = usage_buf;
+        }
+        if (rc == AMS_OK) rc = launch_score_keydiff(p, ctx);
+    }
+    if (rc == AMS_OK && c.pool_kernel > 1 && !split) {
+        rc = launch_smooth_usage(p, p.usage, usage_buf, c.pool_kernel, ctx);
+        p.usage = usage_buf;
+    }
     if (rc == AMS_OK) rc = segment_cluster_supported(p) ? launch_segment_select_cluster(p, ctx) : launch_segment_select(p, ctx);
     if (rc == AMS_OK && dbg) {
         // inspection copies are taken before the table is rewritten
         const size_t U = (size_t)p.L * p.B * p.H;
         cudaError_t e = cudaSuccess;
         if (dbg->scores && e == cudaSuccess) e = cudaMemcpyAsync(dbg->scores, p.scores, U * p.T_cap * 4, cudaMemcpyDeviceToDevice, s);
+        if (dbg->usage && e == cudaSuccess) e = cudaMemcpyAsync(dbg->usage, p.usage, U * p.T_cap * 4, cudaMemcpyDeviceToDevice, s);
         if (dbg->n_segments && e == cudaSuccess) e = cudaMemcpyAsync(dbg->n_segments, p.n_seg, U * 4, cudaMemcpyDeviceToDevice, s);
         if (dbg->seg_bounds && e == cudaSuccess) e = cudaMemcpyAsync(dbg->seg_bounds, p.seg_bounds, U * (size_t)(p.seg_cap + 1) * 4, cudaMemcpyDeviceToDevice, s);
         if (dbg->quotas && e == cudaSuccess) e = cudaMemcpyAsync(dbg->quotas, p.quotas, U * (size_t)p.seg_cap * 4, cudaMemcpyDeviceToDevice, s);
@@ -309,7 +345,7 @@ int ams_get_kernel_times(ams_state *st, float *ms)
 const char *ams_kernel_name(int32_t idx)
 {
     static const char *names[kKernCount] = {"score_phase1", "score_combine", "score_phase2", "segment_select",
-                                            "gather", "table_update"};
+                                            "gather", "table_update", "usage_signal"};
     return idx >= 0 && idx < kKernCount ? names[idx] : nullptr;
 }
 

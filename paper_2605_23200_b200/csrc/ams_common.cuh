@@ -170,7 +170,7 @@ __device__ __forceinline__ uint4 ld_stream16(const void *ptr)
 
 // Host-side launchers (one per translation unit).
 int tova_rows_block(int rows); // query rows handled per pass of the TOVA kernel (8..128)
-enum KernelId { kKernScore1 = 0, kKernScoreCombine, kKernScore2, kKernSegmentSelect, kKernGather, kKernTable, kKernCount };
+enum KernelId { kKernScore1 = 0, kKernScoreCombine, kKernScore2, kKernSegmentSelect, kKernGather, kKernTable, kKernUsage, kKernCount };
 
 // Stream, launch counter and optional per-kernel timing events of one ams_compress call.
 struct LaunchCtx {
@@ -203,5 +203,6 @@ int launch_segment_select(const DevParams &p, LaunchCtx &ctx);
 bool segment_cluster_supported(const DevParams &p);
 int launch_segment_select_cluster(const DevParams &p, LaunchCtx &ctx);
 int launch_gather(const DevParams &p, LaunchCtx &ctx);
+int launch_smooth_usage(const DevParams &p, const float *src, float *dst, int k, LaunchCtx &ctx);
 
 } // namespace ams

@@ -162,11 +162,15 @@ __global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, i
 
     // ---- Eq. 1 weights of this thread's tokens (re-read from shared memory where needed,
     //      so that they do not occupy registers across the reductions)
+    // The usage the mass is built from is the score array itself unless it was smoothed or comes from
+    // another signal; then it is read from global memory (L2) each time.
+    const float *u_sep = p.usage != p.scores ? p.usage + row + t_base : nullptr;
     auto load_w = [&](float (&w)[VPT]) {
 #pragma unroll
         for (int q = 0; q < VPT / 4; ++q) {
             float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-            if (my0 + 4 * q < n_loc) v = *reinterpret_cast<const float4 *>(gs + my0 + 4 * q);
+            if (my0 + 4 * q < n_loc)
+                v = u_sep ? __ldg(reinterpret_cast<const float4 *>(u_sep + my0 + 4 * q)) : *reinterpret_cast<const float4 *>(gs + my0 + 4 * q);
             w[4 * q] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
         }
 #pragma unroll
@@ -802,7 +806,7 @@ constexpr int kNT = 1024;
 // at most eight blocks and the segment tables fit beside the per-token arrays.
 bool segment_cluster_supported(const DevParams &p)
 {
-    if (p.T_cap > 8 * kNT * 16 || p.usage != p.scores) return false;
+    if (p.T_cap > 8 * kNT * 16) return false;
     const int vpt = p.T_cap <= kNT * 4 ? 4 : (p.T_cap <= kNT * 8 ? 8 : 16);
     return smem_map(kNT * vpt, p.seg_cap, p.S, p.beta != 1.0f).total <= (size_t)200 * 1024;
 }

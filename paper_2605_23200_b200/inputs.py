@@ -60,6 +60,8 @@ class Workload:
     steps: int = 1
     append_per_step: int = 0
     resident_layers: int = 0  # 0 = all layers resident
+    pool_kernel: int = 1      # width of the average pooling of the usage scores (1 = none)
+    decoupled: bool = False   # key-only base scores with the window attention as mass signal
 
     @property
     def group(self) -> int:

@@ -26,29 +26,31 @@ class HostSnapshot:
 
 
 def gpu_event(comp: binding.AmsCompressor, cache: inputs.Cache, dst_pages: np.ndarray, scorer_id=None,
-              ext_scores=None, want_dbg=True):
+              ext_scores=None, want_dbg=True, ext_usage=None):
     wl = cache.wl
     dst = torch.from_numpy(dst_pages).to(cache.k_pages.device)
     dbg = comp.make_debug_views(wl.batch, wl.budget) if want_dbg else None
     sid = wl.scorer_id if scorer_id is None else scorer_id
-    q = cache.obs_queries if sid == inputs.SCORER_TOVA else None
+    q = cache.obs_queries if (sid == inputs.SCORER_TOVA or wl.decoupled) else None
     comp.compress(cache.k_pages, cache.v_pages, cache.block_table, cache.seq_lens, q, wl.budget, wl.n_segments,
-                  sid, dst, ext_scores=ext_scores, dbg=dbg)
+                  sid, dst, ext_scores=ext_scores, ext_usage=ext_usage, dbg=dbg)
     comp.status()
     return dbg
 
 
 def compare_event(snap: HostSnapshot, cache: inputs.Cache, comp: binding.AmsCompressor, dbg, dst_pages, credit_before,
-                  scores_for_oracle, units=None, check_bytes=True):
-    """Oracle on `scores_for_oracle` (float32 [L][B][H][T_cap]) must reproduce the library's segments,
-    quotas, keep indices, mass, credit, compacted bytes, block table and lengths exactly."""
+                  scores_for_oracle, units=None, check_bytes=True, usage_for_oracle=None, pool_kernel=1):
+    """Oracle on `scores_for_oracle` (float32 [L][B][H][T_cap]; optionally a separate usage signal, smoothed by
+    the oracle itself with `pool_kernel`) must reproduce the library's segments, quotas, keep indices, mass,
+    credit, compacted bytes, block table and lengths exactly."""
     wl = cache.wl
     prm = params_of(wl)
     k, v = snap.k.copy(), snap.v.copy()
     table, lens = snap.table.copy(), snap.lens.copy()
     credit = credit_before.copy()
     res = oracle.compress(k, v, table, lens, None, credit, wl.budget, prm, oracle.SCORER_EXTERNAL, dst_pages,
-                          ext_scores=scores_for_oracle, units=units, threads=8)
+                          ext_scores=scores_for_oracle, units=units, threads=8, ext_usage=usage_for_oracle,
+                          pool_kernel=pool_kernel)
     n_seg = dbg.n_segments.cpu().numpy()
     bounds = dbg.seg_bounds.cpu().numpy()
     quotas = dbg.quotas.cpu().numpy()

@@ -45,10 +45,19 @@ def test_sizes_and_validation_without_gpu():
         assert lib.ams_segment_capacity(ctypes.byref(cfg)) == want
     cfg = binding.config_for(inputs.CONFIGS[0])
     for field, bad in (("head_dim", 64), ("page_size", 32), ("n_q_heads", 33), ("max_seq_len", 131072 + 16),
-                       ("max_seq_len", 1000), ("eps", 0.0), ("ema_lambda", 1.0), ("ema_beta", 1.5), ("max_budget", 0)):
+                       ("max_seq_len", 1000), ("eps", 0.0), ("ema_lambda", 1.0), ("ema_beta", 1.5), ("max_budget", 0),
+                       ("pool_kernel", 0), ("pool_kernel", 4), ("pool_kernel", 65), ("decoupled", 2)):
         c = binding.config_for(inputs.CONFIGS[0])
         setattr(c, field, bad)
         assert lib.ams_workspace_bytes(ctypes.byref(c)) == 0, field
+    # a smoothed or separate mass signal costs one more per-token array of workspace
+    plain = lib.ams_workspace_bytes(ctypes.byref(cfg))
+    per_token = cfg.n_layers * cfg.max_batch * cfg.n_kv_heads * cfg.max_seq_len * 4
+    for kw in (dict(pool_kernel=5), dict(decoupled=1), dict(pool_kernel=3, decoupled=1)):
+        c = binding.config_for(inputs.CONFIGS[0])
+        for k, v in kw.items():
+            setattr(c, k, v)
+        assert lib.ams_workspace_bytes(ctypes.byref(c)) == plain + per_token
     assert binding.strerror(binding.AMS_ERR_TIMEOUT) == "bounded device wait expired"
     handle = ctypes.c_void_p()
     rc = lib.ams_init_state(ctypes.byref(cfg), None, None, 0, None, ctypes.byref(handle))
