@@ -174,6 +174,20 @@ def run_ours(args, rank, world, local_rank):
         step()
     comp.status()
     torch.cuda.synchronize(dev)
+    direct_step = step
+    if args.graph:
+        # the whole step as one CUDA graph launch (pays off where the step is launch-bound)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            direct_step()
+        restore()
+        step = graph.replay
+        stream = torch.cuda.current_stream(dev)
+        for _ in range(3):
+            restore()
+            step()
+        comp.status()
+        torch.cuda.synchronize(dev)
     barrier()
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -190,7 +204,7 @@ def run_ours(args, rank, world, local_rank):
     acc = {}
     for _ in range(n_prof):
         restore()
-        step()
+        direct_step()
         for k, v in comp.kernel_times_ms().items():
             acc[k] = acc.get(k, 0.0) + v
     comp.set_profiling(False)
@@ -245,7 +259,8 @@ def run_ours(args, rank, world, local_rank):
                    "batch_per_gpu": wl.batch, "cache_tokens": wl.seq_len_max, "budget": wl.budget, "window": wl.window,
                    "n_segments": wl.n_segments, "scorer": "tova" if wl.scorer_id == 0 else "keydiff",
                    "l2": "inputs larger than L2 (K read per step %.2f GB)" % (k_read / 1e9),
-                   "parallelism": f"replica x{world}" if world > 1 else "single GPU"},
+                   "parallelism": f"replica x{world}" if world > 1 else "single GPU",
+                   "launch": "one CUDA graph per step" if args.graph else "direct kernel launches"},
         "effective_hbm_gbs": (k_read + moved) / (ms_per_step * 1e-3) / 1e9,
         "effective_hbm_frac_of_8tbs": (k_read + moved) / (ms_per_step * 1e-3) / 8e12,
         "effective_hbm_frac_of_measured": (k_read + moved) / (ms_per_step * 1e-3) / (peak * 1e9),
@@ -360,6 +375,7 @@ def main():
     ap.add_argument("--config", type=int, default=1)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--graph", action="store_true", help="time the step replayed from a CUDA graph")
     ap.add_argument("--layers", type=int, default=0, help="profiling only: run a reduced layer count")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))

@@ -265,3 +265,45 @@ def test_argument_and_device_errors():
     assert int(lens[0]) == wl.max_seq_len + 16 and int(lens[1]) == wl.budget
     assert comp.status(check=False)[0] == binding.AMS_OK                 # status is cleared by reading it
     assert comp.last_launch_count >= 3
+
+
+def test_event_captured_in_a_cuda_graph_replays_identically():
+    """One event recorded into a CUDA graph (no allocation, no host synchronisation inside the call) and
+    replayed on restored inputs gives the bytes of the directly enqueued event."""
+    wl = _small(1, n_layers=2, batch=2, seq_len_min=1800, seq_len_max=2100, budget=256, window=32)
+    cache = inputs.make_cache(wl, DEV)
+    comp = binding.AmsCompressor(binding.config_for(wl), DEV)
+    dst = torch.from_numpy(inputs.alloc_dst_pages(cache)).to(DEV)
+    table0, lens0 = cache.block_table.clone(), cache.seq_lens.clone()
+    dbg = comp.make_debug_views(wl.batch, wl.budget)
+
+    def restore():
+        cache.block_table.copy_(table0)
+        cache.seq_lens.copy_(lens0)
+        comp.ema_state.zero_()
+
+    def event():
+        comp.compress(cache.k_pages, cache.v_pages, cache.block_table, cache.seq_lens, cache.obs_queries, wl.budget,
+                      wl.n_segments, wl.scorer_id, dst, dbg=dbg)
+
+    event()                                              # direct call (also the warm-up the capture needs)
+    comp.status()
+    want = [t.clone() for t in (dbg.keep_idx, dbg.scores, cache.k_pages, cache.v_pages, cache.block_table,
+                                cache.seq_lens, comp.ema_state)]
+    restore()
+    cache.k_pages[:, dst.reshape(-1).long()] = 0         # the replay must rewrite the replacement pages
+    cache.v_pages[:, dst.reshape(-1).long()] = 0
+    dbg.keep_idx.zero_()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        event()
+    restore()                                            # capture does not execute; state as before the event
+    for _ in range(2):
+        graph.replay()
+        comp.status()
+        got = (dbg.keep_idx, dbg.scores, cache.k_pages, cache.v_pages, cache.block_table, cache.seq_lens, comp.ema_state)
+        for a, b in zip(got, want):
+            assert torch.equal(a.view(torch.int16) if a.dtype == torch.bfloat16 else a,
+                               b.view(torch.int16) if b.dtype == torch.bfloat16 else b)
+        restore()
