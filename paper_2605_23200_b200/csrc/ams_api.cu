@@ -8,7 +8,7 @@
 namespace ams {
 
 struct Layout {
-    size_t status, scores, usage, cbuf, flags, n_seg, seg_bounds, quotas, keep_idx, part, fin, ctrl, finz, total;
+    size_t status, scores, usage, logits, cbuf, flags, n_seg, seg_bounds, quotas, keep_idx, part, fin, ctrl, finz, total;
     int units, T_cap, seg_cap, n_slices, slice_len, rows_pad_cap;
 };
 
@@ -98,6 +98,9 @@ static Layout make_layout(const ams_config *c)
     y.part = off;       off = align_up(off + U * part_per, 256);
     const size_t fin_per = (size_t)((y.rows_pad_cap > kHeadDim ? y.rows_pad_cap : kHeadDim) + 8) * 4;
     y.fin = off;        off = align_up(off + U * fin_per, 256);
+    // narrow query blocks keep their logits (rows_pad floats per token, at most 1/4 of the K bytes) so that
+    // the usage pass need not read K again
+    y.logits = off;     off = align_up(off + (y.rows_pad_cap <= 16 && c->max_window > 0 ? U * T * (size_t)y.rows_pad_cap * 4 : 0), 256);
     y.ctrl = off;       off = align_up(off + U * 2 * 4, 256);
     y.finz = off;       off = align_up(off + U * 128 * 4, 256);
     y.total = off;
@@ -250,6 +253,7 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
     p.fcnt = (int *)(st->ws + y.ctrl);
     p.fflag = p.fcnt + (size_t)c.n_layers * c.max_batch * c.n_kv_heads;
     p.finz = (float *)(st->ws + y.finz);
+    p.logits = (y.rows_pad_cap <= 16 && c.max_window > 0) ? (float *)(st->ws + y.logits) : nullptr;
 
     int rc = AMS_OK;
     LaunchCtx ctx;

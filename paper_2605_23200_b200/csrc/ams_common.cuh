@@ -49,6 +49,7 @@ struct DevParams {
     int tc_tpc_min, tc_stages;        // tensor-core scorer: least tiles per block, K stages in shared memory
     int *fcnt, *fflag;                // fused scorer: per-unit counters of tiles in / of query rows merged ([2][units], contiguous)
     float *finz;                      // fused scorer: 1 / Z_r per unit and query row, [units][rows_pad]
+    float *logits;                    // narrow query blocks (rows_pad <= 16): scaled logits [units][T_cap][rows_pad], or null
     int *status;                      // [4]: code, unit, a, b
 };
 

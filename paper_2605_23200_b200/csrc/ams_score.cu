@@ -7,7 +7,9 @@
 // window.  Two phases over K: phase 1 finds each row's (max, sum of exponentials),
 // phase 2 recomputes the logits and sums the normalised probabilities over rows.
 // The largest probability of a row is 1/Z_r (its arg-max token), so the window
-// maximum is 1/min_r Z_r and needs no third pass.
+// maximum is 1/min_r Z_r and needs no third pass.  With at most 16 (padded) query rows
+// phase 1 also stores the scaled logits (at most 64 bytes per token against the 256
+// bytes of its key), and phase 2 is a per-token kernel over those instead of K.
 //
 // KeyDiff-style score: negative cosine similarity of each key to the mean key of its
 // (sequence, KV head) cache.
@@ -73,6 +75,7 @@ __global__ void __launch_bounds__(kTovaThreads) k_tova(DevParams p)
     const float *fin = p.fin + (size_t)uid * (p.rows_pad + 8);
     float *u_out = p.scores + (size_t)uid * p.T_cap;
     const int n_rb = p.rows_pad / (NTB * 8);
+    float *lg = (PHASE == 1 && p.logits && n_rb == 1) ? p.logits + (size_t)uid * p.T_cap * (NTB * 8) : nullptr;
     const float pmax = PHASE == 2 ? fin[p.rows_pad] : 0.0f;
     const float inv_rows = 1.0f / (float)p.rows;
 
@@ -131,12 +134,14 @@ __global__ void __launch_bounds__(kTovaThreads) k_tova(DevParams p)
                     mma_bf16(d, x[j].x, y[j].x, x[j].y, y[j].y, zq[j].x, zq[j].y);
                     mma_bf16(d, x[j].z, y[j].z, x[j].w, y[j].w, zq[j].z, zq[j].w);
                 }
+                float keep_a[2], keep_b[2];
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
                     const int lv = min(lastv[nt][e], t_end - 1);
                     const float va = ta <= lv ? d[e] * c : -INFINITY;
                     const float vb = tb <= lv ? d[2 + e] * c : -INFINITY;
                     if (PHASE == 1) {
+                        if (NTB <= 2) { keep_a[e] = va; keep_b[e] = vb; }
                         const float mn = fmaxf(st_a[nt][e], fmaxf(va, vb));
                         if (mn != -INFINITY) {
                             st_b[nt][e] = st_b[nt][e] * ex2(st_a[nt][e] - mn) + ex2(va - mn) + ex2(vb - mn);
@@ -146,6 +151,10 @@ __global__ void __launch_bounds__(kTovaThreads) k_tova(DevParams p)
                         acc_a += ex2(va - st_a[nt][e]);
                         acc_b += ex2(vb - st_a[nt][e]);
                     }
+                }
+                if (PHASE == 1 && NTB <= 2 && lg) { // pairs the window hides are stored as -inf: they add nothing later
+                    if (ta < t_end) *reinterpret_cast<float2 *>(lg + (size_t)ta * (NTB * 8) + nt * 8 + 2 * tq) = make_float2(keep_a[0], keep_a[1]);
+                    if (tb < t_end) *reinterpret_cast<float2 *>(lg + (size_t)tb * (NTB * 8) + nt * 8 + 2 * tq) = make_float2(keep_b[0], keep_b[1]);
                 }
             }
             if (PHASE == 2) {
@@ -227,6 +236,36 @@ __global__ void __launch_bounds__(128) k_tova_combine(DevParams p)
     }
     best = block_max_f32(best, scratch);
     if (threadIdx.x == 0) fin[p.rows_pad] = best;
+}
+
+// Usage pass over stored logits (RP = padded query rows, 8 or 16): one thread per token sums
+// 2^(x_r - b_r) over the rows; pairs the window hides were stored as -inf, padding rows have
+// b_r = +inf; the hidden pairs count as the window maximum.
+template <int RP>
+__global__ void __launch_bounds__(256) k_tova_usage_from_logits(DevParams p)
+{
+    __shared__ float bs[RP + 1];
+    const int uid = blockIdx.x;
+    const int b = (uid / p.H) % p.B;
+    const int T = p.seq_lens[b];
+    if (T <= p.Tk || T > p.T_cap || p.W > T) return;
+    const float *fin = p.fin + (size_t)uid * (p.rows_pad + 8);
+    if (threadIdx.x <= RP) bs[threadIdx.x] = fin[threadIdx.x]; // b_r of the rows, then the window maximum
+    __syncthreads();
+    const int t = blockIdx.y * 256 + threadIdx.x;
+    if (t >= T) return;
+    const float4 *x = reinterpret_cast<const float4 *>(p.logits + ((size_t)uid * p.T_cap + t) * RP);
+    float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+    for (int q = 0; q < RP / 4; ++q) {
+        const float4 v = __ldcs(x + q);
+        acc[0] += ex2(v.x - bs[4 * q]);
+        acc[1] += ex2(v.y - bs[4 * q + 1]);
+        acc[2] += ex2(v.z - bs[4 * q + 2]);
+        acc[3] += ex2(v.w - bs[4 * q + 3]);
+    }
+    const int ninv = p.causal ? p.G * max(0, t - (T - p.W)) : 0;
+    p.scores[(size_t)uid * p.T_cap + t] = ((acc[0] + acc[1]) + (acc[2] + acc[3]) + (float)ninv * bs[RP]) * (1.0f / (float)p.rows);
 }
 
 // ---------------------------------------------------------------------------- KeyDiff
@@ -329,7 +368,12 @@ void launch_tova_ntb(const DevParams &p, LaunchCtx &ctx)
     ctx.mark(kKernScore1);
     k_tova_combine<<<p.L * p.B * p.H, 128, 0, ctx.s>>>(p);
     ctx.mark(kKernScoreCombine);
-    k_tova<NTB, 2><<<grid, kTovaThreads, 0, ctx.s>>>(p);
+    if (NTB <= 2 && p.logits && p.rows_pad == NTB * 8) {
+        const dim3 g2(p.L * p.B * p.H, (p.T_cap + 255) / 256);
+        k_tova_usage_from_logits<NTB * 8><<<g2, 256, 0, ctx.s>>>(p);
+    } else {
+        k_tova<NTB, 2><<<grid, kTovaThreads, 0, ctx.s>>>(p);
+    }
     ctx.mark(kKernScore2);
 }
 
