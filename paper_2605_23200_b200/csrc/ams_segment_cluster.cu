@@ -61,7 +61,7 @@ __host__ __device__ inline SmemMap smem_map(int tpc, int sc, int S, bool ema_on)
 }
 
 template <int NT, int VPT>
-__global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, int cs)
+__global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, int cs, int cs_max)
 {
     constexpr int nt = NT, TPC = NT * VPT;
     extern __shared__ __align__(16) unsigned char dyn[];
@@ -76,7 +76,9 @@ __global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, i
     const int T = p.seq_lens[b];
     // every exit below is taken by all blocks of the cluster together
     if (T <= p.Tk) return; // nothing to evict
-    if (T > p.T_cap) { if (tid == 0 && rank == 0) set_status(p.status, AMS_ERR_CAPACITY, uid, T, p.T_cap); return; }
+    if (T > p.T_cap) { if (tid == 0 && rank == 0 && cs == cs_max) set_status(p.status, AMS_ERR_CAPACITY, uid, T, p.T_cap); return; }
+    // one launch per cluster size: this one takes the sequences that need exactly cs blocks
+    if (T > cs * TPC || (cs > 1 && T <= (cs / 2) * TPC)) return;
 
     const int sc = p.seg_cap;
     const bool ema_on = p.beta != 1.0f;
@@ -771,7 +773,7 @@ __global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, i
 }
 
 template <int NT, int VPT>
-int launch_cfg(const DevParams &p, LaunchCtx &ctx, int cs, size_t smem)
+int launch_cfg(const DevParams &p, LaunchCtx &ctx, int cs, int cs_max, size_t smem)
 {
     static size_t configured = 0;
     if (smem > configured) {
@@ -793,7 +795,7 @@ int launch_cfg(const DevParams &p, LaunchCtx &ctx, int cs, size_t smem)
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, k_segment_select_cluster<NT, VPT>, p, cs) != cudaSuccess) return AMS_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, k_segment_select_cluster<NT, VPT>, p, cs, cs_max) != cudaSuccess) return AMS_ERR_CUDA;
     ctx.mark(kKernSegmentSelect);
     return AMS_OK;
 }
@@ -814,13 +816,21 @@ bool segment_cluster_supported(const DevParams &p)
 int launch_segment_select_cluster(const DevParams &p, LaunchCtx &ctx)
 {
     const bool ema_on = p.beta != 1.0f;
-    if (p.T_cap <= kNT * 4) return launch_cfg<kNT, 4>(p, ctx, 1, smem_map(kNT * 4, p.seg_cap, p.S, ema_on).total);
-    if (p.T_cap <= kNT * 8) return launch_cfg<kNT, 8>(p, ctx, 1, smem_map(kNT * 8, p.seg_cap, p.S, ema_on).total);
+    if (p.T_cap <= kNT * 4) return launch_cfg<kNT, 4>(p, ctx, 1, 1, smem_map(kNT * 4, p.seg_cap, p.S, ema_on).total);
+    if (p.T_cap <= kNT * 8) return launch_cfg<kNT, 8>(p, ctx, 1, 1, smem_map(kNT * 8, p.seg_cap, p.S, ema_on).total);
     const int tpc = kNT * 16;
     const int cs_need = (p.T_cap + tpc - 1) / tpc;
-    int cs = 1;
-    while (cs < cs_need) cs *= 2; // cluster sizes are powers of two
-    return launch_cfg<kNT, 16>(p, ctx, cs, smem_map(tpc, p.seg_cap, p.S, ema_on).total);
+    int cs_max = 1;
+    while (cs_max < cs_need) cs_max *= 2; // cluster sizes are powers of two
+    // Sequence lengths are known on the device only: one launch per cluster size, each taking the
+    // sequences that need exactly that many blocks (the blocks of the others leave at once), so that a
+    // short sequence of a ragged batch does not pay for the cluster barriers of the longest one.
+    const size_t smem = smem_map(tpc, p.seg_cap, p.S, ema_on).total;
+    for (int cs = 1; cs <= cs_max; cs *= 2) {
+        const int rc = launch_cfg<kNT, 16>(p, ctx, cs, cs_max, smem);
+        if (rc != AMS_OK) return rc;
+    }
+    return AMS_OK;
 }
 
 } // namespace ams
