@@ -5,16 +5,18 @@
 // takes the contiguous tile range [c * tpc, (c + 1) * tpc).  Inside a block:
 //   warp 0      TMA producer: query block of the current unit, then one 32 KB K tile per
 //               stage (eight 16-token pages, one 4 KB copy each, 128-byte swizzle);
-//   warps 1, 3  MMA issuers (one lane each, one per consumer warpgroup, tiles in turn): per
-//               (tile, 128-row query block) eight
-//               tcgen05.mma m128 n128 k16 into one of four 128-column TMEM slots (two per
-//               consumer warpgroup, used in turn);
-//   warps 4-11  two consumer warpgroups, alternating tiles; thread i of a warpgroup owns
-//               TMEM lane i of its slots.
+//   warps 1, 3  MMA issuers (one lane each, one per pair of consumer warpgroups, tiles in
+//               turn): per (tile, 128-row query block) eight tcgen05.mma m128 n128 k16 into
+//               one of four 128-column TMEM slots (two per pair, used in turn);
+//   warps 4-19  four consumer warpgroups in two pairs, the pairs alternating tiles; thread i
+//               of either warpgroup of a pair owns TMEM lane i of the pair's slots, the
+//               first warpgroup taking columns [0, 64) and the second [64, 128).  (Two
+//               warpgroups alone left each scheduler with two dependent instruction streams
+//               and the accumulators waiting for them; four hide that latency.)
 // Phase 1 puts query rows on the TMEM lanes (A = Q, B = K), so a thread folds its row's
 // logits into a running (max, sum of 2^x) without leaving registers; phase 2 puts tokens
 // on the lanes (A = K, B = Q), so a thread sums 2^(x - b_r) over the query rows of its
-// token.  Both operands are K-major 128-byte-swizzled tiles, so the same shared-memory
+// token (the two halves of the rows meet through shared memory).  Both operands are K-major 128-byte-swizzled tiles, so the same shared-memory
 // tiles serve either role.  Every wait is bounded; on expiry the block reports
 // AMS_ERR_TIMEOUT, drains its copies, frees its TMEM and returns.
 #include <cuda.h>
@@ -28,7 +30,8 @@ using namespace tc;
 
 namespace {
 
-constexpr int kTcThreads = 384;
+constexpr int kTcThreads = 640;
+constexpr int kConsumerThreads = 512;                // warps 4-19
 constexpr int kTileTokens = 128;
 constexpr int kTileBytes = kTileTokens * kRowBytes;  // 32 KB
 constexpr int kHalfBytes = kTileBytes / 2;           // one 64-wide half of a 128-row tile
@@ -38,9 +41,11 @@ constexpr int kMaxStages = 6;
 struct TcShared {
     unsigned long long kfull[kMaxStages], kempty[kMaxStages], tfull[kSlots], tempty[kSlots];
     unsigned long long qfull, qempty, done[2];
+    unsigned long long pfull[2][2];                  // usage pass: second half's partial sums are in pacc[pair][slot bit]
+    float pacc[2][2][128];
     uint32_t tmem_base;
     int abort_flag;
-    float wmax[2][8];
+    float wmax[2][16];
     int tiles_lh, tpc;
     long long n_tiles;
 };
@@ -103,12 +108,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
     unsigned char *Qs = base;                                   // [n_rb][2 halves][128 rows][128 B]
     unsigned char *Ks = Qs + (size_t)n_rb * kTileBytes;         // [NS][2 halves][128 rows][128 B]
     float *fin_s = reinterpret_cast<float *>(Ks + (size_t)NS * kTileBytes);   // [2][rows_pad]
-    float2 *red = reinterpret_cast<float2 *>(fin_s + 2 * p.rows_pad);         // [2][n_rb][128]
+    float2 *red = reinterpret_cast<float2 *>(fin_s + 2 * p.rows_pad);         // [3][n_rb][128]
     volatile int *abort_flag = &sh.abort_flag;
 
     if (tid == 0) {
         for (int i = 0; i < kMaxStages; ++i) { mbar_init(smem_u32(&sh.kfull[i]), 1); mbar_init(smem_u32(&sh.kempty[i]), 1); }
-        for (int i = 0; i < kSlots; ++i) { mbar_init(smem_u32(&sh.tfull[i]), 1); mbar_init(smem_u32(&sh.tempty[i]), 4); }
+        for (int i = 0; i < kSlots; ++i) { mbar_init(smem_u32(&sh.tfull[i]), 1); mbar_init(smem_u32(&sh.tempty[i]), 8); }
+        for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&sh.pfull[i >> 1][i & 1]), 4);
         mbar_init(smem_u32(&sh.qfull), 1);
         mbar_init(smem_u32(&sh.qempty), 2); // both MMA issuers release the query block
         mbar_init(smem_u32(&sh.done[0]), 1);
@@ -184,11 +190,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
             }
         } else if (warp == 1 || warp == 3) {
             // ------------------------------------------------------------ MMA issuers
-            // One thread per consumer warpgroup, taking the tiles in turn: a tile costs its issuer a
+            // One thread per consumer pair, taking the tiles in turn: a tile costs its issuer a
             // chain of long waits (two barriers, eight MMAs, two commits) that is longer than the
             // tile's share of the HBM stream, so a single issuer would be the bottleneck.
             if (lane == 0) {
-                const int wg = warp >> 1; // issuer 0 feeds warpgroup 0 (even tiles), issuer 1 warpgroup 1
+                const int wg = warp >> 1; // issuer 0 feeds consumer pair 0 (even tiles), issuer 1 pair 1
                 int kit = 0, seg = 0, wsit = 0; // wsit: accumulator slots handed to the warpgroup so far
                 bool ok = true;
                 for (long long g = g_begin; g < g_end && ok;) {
@@ -228,8 +234,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
             __syncwarp();
         } else if (warp >= 4) {
             // ------------------------------------------------------------ consumers
-            const int wg = (warp - 4) >> 2, quad = warp & 3, li = quad * 32 + lane; // li = TMEM lane of this thread
-            int kit = 0, wsit = 0, seg = 0;
+            // Four warpgroups.  Warpgroups (pair, 0) and (pair, 1) share the tiles of one pair (tiles in
+            // turn between the two pairs): thread li of either owns TMEM lane li, the first takes
+            // columns [0, 64) of the slot and the second columns [64, 128).
+            const int wgq = (warp - 4) >> 2, pair = wgq & 1, half = wgq >> 1, quad = warp & 3, li = quad * 32 + lane;
+            int kit = 0, wsit = 0, seg = 0, pc0 = 0, pc1 = 0; // pc*: uses so far of this pair's two hand-over barriers
             bool ok = true;
             // a thread whose wait ran out keeps walking the segments without touching the pipeline, so that
             // the consumers' named barriers stay matched
@@ -254,7 +263,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
                     const long long ustart = g - s.tile0;
                     const int n_parts = (int)((ustart + nt_u - 1) / tpc) - (int)(ustart / tpc) + 1;
                     float best = 0.0f;
-                    for (int r = (warp - 4) * 32 + lane; r < p.rows_pad; r += 256) {
+                    for (int r = (warp - 4) * 32 + lane; r < p.rows_pad; r += kConsumerThreads) {
                         float mm = -INFINITY, zz = 0.0f;
                         for (int q = 0; q < n_parts; ++q) {
                             const float2 v = __ldcg(reinterpret_cast<const float2 *>(p.part) + ((size_t)s.uid * p.n_slices + q) * p.rows_pad + r);
@@ -267,116 +276,143 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
 #pragma unroll
                     for (int o = 16; o > 0; o >>= 1) best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, o));
                     if (lane == 0) sh.wmax[seg & 1][warp - 4] = best;
-                    asm volatile("bar.sync 1, 256;" ::: "memory");
+                    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
 #pragma unroll
-                    for (int w = 0; w < 8; ++w) pmax = fmaxf(pmax, sh.wmax[seg & 1][w]);
+                    for (int w = 0; w < kConsumerThreads / 32; ++w) pmax = fmaxf(pmax, sh.wmax[seg & 1][w]);
                 }
                 for (int i = 0; i < s.n && ok; ++i, ++kit) {
-                    if ((kit & 1) != wg) continue;
+                    if ((kit & 1) != pair) continue;
                     const int t0 = (s.tile0 + i) * kTileTokens;
                     float acc = 0.0f;
+                    int last_slot = 0;
                     for (int rb = 0; rb < n_rb && ok; ++rb, ++wsit) {
-                        const int slot = 2 * wg + (wsit & 1);
+                        const int slot = 2 * pair + (wsit & 1);
+                        last_slot = slot;
                         ok = mbar_wait(smem_u32(&sh.tfull[slot]), (uint32_t)((wsit >> 1) & 1), abort_flag);
                         if (!ok) break;
                         tc_fence_after();
-                        const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * 128);
-                        // chunks of 32 columns, the load of the next chunk in flight while this one is worked on
-                        uint32_t buf[2][32];
-                        tc_ld32_issue(taddr, buf[0]);
-                        tc_ld_wait(buf[0]);
+                        const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * 128 + half * 64);
+                        // chunks of 16 columns, the load of the next chunk in flight while this one is worked on
+                        uint32_t buf[2][16];
+                        tc_ld16_issue(taddr, buf[0]);
+                        tc_ld16_wait(buf[0]);
                         if (PHASE == 1) {
                             const int lv = min(lastv[rb], T - 1);
                             float mr = m[rb], zr = z[rb];
 #pragma unroll
                             for (int ch = 0; ch < 4; ++ch) {
-                                uint32_t (&cur)[32] = buf[ch & 1];
-                                if (ch < 3) tc_ld32_issue(taddr + (ch + 1) * 32, buf[(ch + 1) & 1]);
-                                const int tc0 = t0 + ch * 32;
+                                uint32_t (&cur)[16] = buf[ch & 1];
+                                if (ch < 3) tc_ld16_issue(taddr + (ch + 1) * 16, buf[(ch + 1) & 1]);
+                                const int tc0 = t0 + half * 64 + ch * 16;
                                 if (tc0 <= lv) {
-                                    float v[32];
+                                    float v[16];
 #pragma unroll
-                                    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(cur[j]);
-                                    if (tc0 + 31 > lv) {
+                                    for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(cur[j]);
+                                    if (tc0 + 15 > lv) {
 #pragma unroll
-                                        for (int j = 0; j < 32; ++j) if (tc0 + j > lv) v[j] = -INFINITY;
+                                        for (int j = 0; j < 16; ++j) if (tc0 + j > lv) v[j] = -INFINITY;
                                     }
-                                    // tree of three-input maxima: depth 4 instead of a chain of 31
-                                    float a8[8];
+                                    // tree of three-input maxima instead of a chain of 15
+                                    float a5[5];
 #pragma unroll
-                                    for (int j = 0; j < 8; ++j) a8[j] = max3(v[j], v[j + 8], v[j + 16]);
-#pragma unroll
-                                    for (int j = 0; j < 8; ++j) a8[j] = fmaxf(a8[j], v[j + 24]);
-                                    const float cm = fmaxf(max3(a8[0], a8[1], a8[2]), fmaxf(max3(a8[3], a8[4], a8[5]), fmaxf(a8[6], a8[7])));
+                                    for (int j = 0; j < 5; ++j) a5[j] = max3(v[j], v[j + 5], v[j + 10]);
+                                    const float cm = fmaxf(max3(a5[0], a5[1], a5[2]), max3(a5[3], a5[4], v[15]));
                                     const float mn = fmaxf(mr, cm * c);
                                     zr *= ex2(mr - mn);
                                     mr = mn;
                                     float zs[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
-                                    for (int j = 0; j < 32; ++j) zs[j & 3] += ex2(fmaf(v[j], c, -mn));
+                                    for (int j = 0; j < 16; ++j) zs[j & 3] += ex2(fmaf(v[j], c, -mn));
                                     zr += (zs[0] + zs[1]) + (zs[2] + zs[3]);
                                 }
-                                if (ch < 3) tc_ld_wait(buf[(ch + 1) & 1]);
+                                if (ch < 3) tc_ld16_wait(buf[(ch + 1) & 1]);
                             }
                             m[rb] = mr; z[rb] = zr;
                         } else {
                             const int t = t0 + li;
                             const bool plain = !p.causal || t0 + kTileTokens - 1 <= T - p.W;
-                            const float4 *fr4 = reinterpret_cast<const float4 *>(fs + rb * 128);
+                            const float4 *fr4 = reinterpret_cast<const float4 *>(fs + rb * 128 + half * 64);
                             float ac[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
                             for (int ch = 0; ch < 4; ++ch) {
-                                uint32_t (&cur)[32] = buf[ch & 1];
-                                if (ch < 3) tc_ld32_issue(taddr + (ch + 1) * 32, buf[(ch + 1) & 1]);
+                                uint32_t (&cur)[16] = buf[ch & 1];
+                                if (ch < 3) tc_ld16_issue(taddr + (ch + 1) * 16, buf[(ch + 1) & 1]);
                                 if (plain) {
 #pragma unroll
-                                    for (int j4 = 0; j4 < 8; ++j4) {
-                                        const float4 f = fr4[ch * 8 + j4];
+                                    for (int j4 = 0; j4 < 4; ++j4) {
+                                        const float4 f = fr4[ch * 4 + j4];
                                         ac[0] += ex2(fmaf(__uint_as_float(cur[4 * j4]), c, -f.x));
                                         ac[1] += ex2(fmaf(__uint_as_float(cur[4 * j4 + 1]), c, -f.y));
                                         ac[2] += ex2(fmaf(__uint_as_float(cur[4 * j4 + 2]), c, -f.z));
                                         ac[3] += ex2(fmaf(__uint_as_float(cur[4 * j4 + 3]), c, -f.w));
                                     }
                                 } else {
-                                    const int rbase = rb * 128 + ch * 32;
+                                    const int rbase = rb * 128 + half * 64 + ch * 16;
 #pragma unroll
-                                    for (int j = 0; j < 32; ++j) {
+                                    for (int j = 0; j < 16; ++j) {
                                         const int r = rbase + j;
                                         const bool seen = t <= T - p.W + (r % p.W);
                                         ac[j & 3] += seen ? ex2(fmaf(__uint_as_float(cur[j]), c, -fs[r])) : 0.0f;
                                     }
                                 }
-                                if (ch < 3) tc_ld_wait(buf[(ch + 1) & 1]);
+                                if (ch < 3) tc_ld16_wait(buf[(ch + 1) & 1]);
                             }
                             acc += (ac[0] + ac[1]) + (ac[2] + ac[3]);
                         }
+                        if (PHASE == 2 && rb == n_rb - 1) break; // the slot of a tile's last query block is released below
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(smem_u32(&sh.tempty[slot]));
                     }
                     if (PHASE == 2 && ok) {
-                        const int t = t0 + li;
-                        if (t < T) {
-                            const int ninv = p.causal ? p.G * max(0, t - (T - p.W)) : 0;
-                            p.scores[(size_t)s.uid * p.T_cap + t] = (acc + (float)ninv * pmax) * (1.0f / (float)p.rows);
+                        // The two halves of the query rows meet here: the second warpgroup leaves its sum in shared
+                        // memory, the first adds it and writes the token's usage.  The buffer is the one of the slot,
+                        // and the first warpgroup releases the slot only after reading it, so the next tile that
+                        // maps to this slot cannot overwrite it early.
+                        ++wsit; // (the loop above left through its break)
+                        const int bit = last_slot & 1;
+                        float *pa = sh.pacc[pair][bit];
+                        const uint32_t pbar = smem_u32(&sh.pfull[pair][bit]);
+                        if (half == 1) {
+                            pa[li] = acc;
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) { mbar_arrive(pbar); mbar_arrive(smem_u32(&sh.tempty[last_slot])); }
+                        } else {
+                            ok = mbar_wait(pbar, (uint32_t)((bit ? pc1 : pc0) & 1), abort_flag);
+                            if (ok) {
+                                acc += pa[li];
+                                const int t = t0 + li;
+                                if (t < T) {
+                                    const int ninv = p.causal ? p.G * max(0, t - (T - p.W)) : 0;
+                                    p.scores[(size_t)s.uid * p.T_cap + t] = (acc + (float)ninv * pmax) * (1.0f / (float)p.rows);
+                                }
+                                tc_fence_before();
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(smem_u32(&sh.tempty[last_slot]));
+                            }
                         }
+                        if (bit) ++pc1; else ++pc0;
                     }
                 }
                 if (PHASE == 1) {
-                    // fold the two warpgroups' statistics and store this block's part of the unit
-                    float2 *rd = red + (size_t)(seg & 1) * n_rb * 128;
-                    if (wg == 1)
-                        for (int rb = 0; rb < n_rb; ++rb) rd[rb * 128 + li] = make_float2(m[rb], z[rb]);
-                    asm volatile("bar.sync 1, 256;" ::: "memory");
-                    if (wg == 0 && ok) {
+                    // fold the four warpgroups' statistics (fixed order) and store this block's part of the unit
+                    float2 *rd = red;
+                    if (wgq > 0)
+                        for (int rb = 0; rb < n_rb; ++rb) rd[((wgq - 1) * n_rb + rb) * 128 + li] = make_float2(m[rb], z[rb]);
+                    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
+                    if (wgq == 0 && ok) {
                         float2 *out = reinterpret_cast<float2 *>(p.part) + ((size_t)s.uid * p.n_slices + s.part) * p.rows_pad;
                         for (int rb = 0; rb < n_rb; ++rb) {
-                            const float2 o = rd[rb * 128 + li];
                             float mm = m[rb], zz = z[rb];
-                            lse_merge(mm, zz, o.x, o.y);
+                            for (int w = 0; w < 3; ++w) {
+                                const float2 o = rd[(w * n_rb + rb) * 128 + li];
+                                lse_merge(mm, zz, o.x, o.y);
+                            }
                             out[rb * 128 + li] = make_float2(mm, zz);
                         }
                     }
+                    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory"); // the buffer is free again
                 }
                 g += s.n;
                 ++seg;
@@ -398,7 +434,7 @@ bool tova_tc_supported(const DevParams &p) { return p.rows >= 64 && p.rows_pad %
 size_t tova_tc_smem_bytes(const DevParams &p)
 {
     return 1024 + (size_t)(p.rows_pad / 128 + p.tc_stages) * kTileBytes + (size_t)2 * p.rows_pad * 4 +
-           (size_t)2 * (p.rows_pad / 128) * 128 * 8 + 256;
+           (size_t)3 * (p.rows_pad / 128) * 128 * 8 + 256;
 }
 
 int launch_score_tova_tc(const DevParams &p, LaunchCtx &ctx)
