@@ -60,10 +60,12 @@ __host__ __device__ inline SmemMap smem_map(int tpc, int sc, int S, bool ema_on)
     return m;
 }
 
-template <int NT, int VPT>
-__global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, int cs, int cs_max)
+// CS (blocks per cluster) is a template parameter so that every loop over the ranks of the cluster
+// unrolls into independent remote loads instead of a chain of dependent ones.
+template <int NT, int VPT, int CS>
+__global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, int cs_max)
 {
-    constexpr int nt = NT, TPC = NT * VPT;
+    constexpr int nt = NT, TPC = NT * VPT, cs = CS;
     extern __shared__ __align__(16) unsigned char dyn[];
     __shared__ Smem sm;
     __shared__ u64 xch[kXch];
@@ -123,6 +125,7 @@ __global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, i
         if (tid == 0) *slot = mine;
         cluster.sync();
         u64 tot = 0;
+#pragma unroll
         for (int r = 0; r < cs; ++r) {
             const u64 x = *cluster.map_shared_rank(slot, r);
             if (prefix && r < rank) *prefix += x;
@@ -137,6 +140,7 @@ __global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, i
         if (tid == 0) *slot = (u64)__float_as_uint(mine);
         cluster.sync();
         float m = mine;
+#pragma unroll
         for (int r = 0; r < cs; ++r) m = fmaxf(m, __uint_as_float((unsigned)*cluster.map_shared_rank(slot, r)));
         return m;
     };
@@ -502,6 +506,7 @@ __global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, i
                 int a1 = c[sg * 3], a2 = c[sg * 3 + 1], a3 = c[sg * 3 + 2];
                 if (cs > 1) {
                     a1 = a2 = a3 = 0;
+#pragma unroll
                     for (int r = 0; r < cs; ++r) {
                         const int *rc = cluster.map_shared_rank(c + sg * 3, r);
                         a1 += rc[0]; a2 += rc[1]; a3 += rc[2];
@@ -690,7 +695,10 @@ __global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, i
             unit_barrier();
             int v = 0;
             if (cs == 1) v = lane < nwarps ? mine[lane] : 0;
-            else for (int r = 0; r < cs; ++r) v += lane < nwarps ? cluster.map_shared_rank(mine, r)[lane] : 0;
+            else {
+#pragma unroll
+                for (int r = 0; r < cs; ++r) v += lane < nwarps ? cluster.map_shared_rank(mine, r)[lane] : 0;
+            }
             return __reduce_add_sync(0xffffffffu, v);
         };
         unsigned P = 0;
@@ -772,30 +780,30 @@ __global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, i
     if (cs > 1) cluster.sync(); // nobody leaves while a neighbour may still read its shared memory
 }
 
-template <int NT, int VPT>
-int launch_cfg(const DevParams &p, LaunchCtx &ctx, int cs, int cs_max, size_t smem)
+template <int NT, int VPT, int CS>
+int launch_cfg(const DevParams &p, LaunchCtx &ctx, int cs_max, size_t smem)
 {
     static size_t configured = 0;
     if (smem > configured) {
-        if (cudaFuncSetAttribute(k_segment_select_cluster<NT, VPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        if (cudaFuncSetAttribute(k_segment_select_cluster<NT, VPT, CS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return AMS_ERR_CUDA;
         configured = smem;
     }
     const int units = p.L * p.B * p.H;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
-    cfg.gridDim = dim3((unsigned)(units * cs), 1, 1);
+    cfg.gridDim = dim3((unsigned)(units * CS), 1, 1);
     cfg.blockDim = dim3(NT, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = ctx.s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)cs;
+    attr[0].val.clusterDim.x = (unsigned)CS;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, k_segment_select_cluster<NT, VPT>, p, cs, cs_max) != cudaSuccess) return AMS_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, k_segment_select_cluster<NT, VPT, CS>, p, cs_max) != cudaSuccess) return AMS_ERR_CUDA;
     ctx.mark(kKernSegmentSelect);
     return AMS_OK;
 }
@@ -816,8 +824,8 @@ bool segment_cluster_supported(const DevParams &p)
 int launch_segment_select_cluster(const DevParams &p, LaunchCtx &ctx)
 {
     const bool ema_on = p.beta != 1.0f;
-    if (p.T_cap <= kNT * 4) return launch_cfg<kNT, 4>(p, ctx, 1, 1, smem_map(kNT * 4, p.seg_cap, p.S, ema_on).total);
-    if (p.T_cap <= kNT * 8) return launch_cfg<kNT, 8>(p, ctx, 1, 1, smem_map(kNT * 8, p.seg_cap, p.S, ema_on).total);
+    if (p.T_cap <= kNT * 4) return launch_cfg<kNT, 4, 1>(p, ctx, 1, smem_map(kNT * 4, p.seg_cap, p.S, ema_on).total);
+    if (p.T_cap <= kNT * 8) return launch_cfg<kNT, 8, 1>(p, ctx, 1, smem_map(kNT * 8, p.seg_cap, p.S, ema_on).total);
     const int tpc = kNT * 16;
     const int cs_need = (p.T_cap + tpc - 1) / tpc;
     int cs_max = 1;
@@ -826,11 +834,11 @@ int launch_segment_select_cluster(const DevParams &p, LaunchCtx &ctx)
     // sequences that need exactly that many blocks (the blocks of the others leave at once), so that a
     // short sequence of a ragged batch does not pay for the cluster barriers of the longest one.
     const size_t smem = smem_map(tpc, p.seg_cap, p.S, ema_on).total;
-    for (int cs = 1; cs <= cs_max; cs *= 2) {
-        const int rc = launch_cfg<kNT, 16>(p, ctx, cs, cs_max, smem);
-        if (rc != AMS_OK) return rc;
-    }
-    return AMS_OK;
+    int rc = launch_cfg<kNT, 16, 1>(p, ctx, cs_max, smem);
+    if (rc == AMS_OK && cs_max >= 2) rc = launch_cfg<kNT, 16, 2>(p, ctx, cs_max, smem);
+    if (rc == AMS_OK && cs_max >= 4) rc = launch_cfg<kNT, 16, 4>(p, ctx, cs_max, smem);
+    if (rc == AMS_OK && cs_max >= 8) rc = launch_cfg<kNT, 16, 8>(p, ctx, cs_max, smem);
+    return rc;
 }
 
 } // namespace ams
