@@ -8,7 +8,7 @@
 namespace ams {
 
 struct Layout {
-    size_t status, scores, usage, logits, cbuf, flags, n_seg, seg_bounds, quotas, keep_idx, part, fin, ctrl, finz, total;
+    size_t status, scores, usage, logits, qctrl, cbuf, flags, n_seg, seg_bounds, quotas, keep_idx, part, fin, ctrl, finz, total;
     int units, T_cap, seg_cap, n_slices, slice_len, rows_pad_cap;
 };
 
@@ -102,6 +102,7 @@ static Layout make_layout(const ams_config *c)
     // the usage pass need not read K again
     y.logits = off;     off = align_up(off + (y.rows_pad_cap <= 16 && c->max_window > 0 ? U * T * (size_t)y.rows_pad_cap * 4 : 0), 256);
     y.ctrl = off;       off = align_up(off + U * 2 * 4, 256);
+    y.qctrl = off;      off = align_up(off + (size_t)(4 + c->n_layers * c->max_batch) * 4, 256);
     y.finz = off;       off = align_up(off + U * 128 * 4, 256);
     y.total = off;
     return y;
@@ -253,6 +254,7 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
     p.fcnt = (int *)(st->ws + y.ctrl);
     p.fflag = p.fcnt + (size_t)c.n_layers * c.max_batch * c.n_kv_heads;
     p.finz = (float *)(st->ws + y.finz);
+    p.qctrl = (int *)(st->ws + y.qctrl);
     p.logits = (y.rows_pad_cap <= 16 && c.max_window > 0) ? (float *)(st->ws + y.logits) : nullptr;
 
     int rc = AMS_OK;
@@ -282,6 +284,7 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
         rc = launch_smooth_usage(p, p.usage, usage_buf, c.pool_kernel, ctx);
         p.usage = usage_buf;
     }
+    const bool queued = segment_moves_rows(p); // the work-queue form of the segmentation kernel starts the compaction
     if (rc == AMS_OK) rc = segment_cluster_supported(p) ? launch_segment_select_cluster(p, ctx) : launch_segment_select(p, ctx);
     if (rc == AMS_OK && dbg) {
         // inspection copies are taken before the table is rewritten
@@ -295,7 +298,7 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
         if (dbg->keep_idx && e == cudaSuccess) e = cudaMemcpyAsync(dbg->keep_idx, p.keep_idx, U * (size_t)p.Tk * 4, cudaMemcpyDeviceToDevice, s);
         if (e != cudaSuccess) rc = AMS_ERR_CUDA;
     }
-    if (rc == AMS_OK) rc = launch_gather(p, ctx);
+    if (rc == AMS_OK) rc = launch_gather(p, ctx, queued);
     st->last_launches = ctx.launches;
     st->n_ev = ctx.n_ev;
     memcpy(st->ev_ids, ctx.ids, sizeof ctx.ids);

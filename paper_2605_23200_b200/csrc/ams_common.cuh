@@ -49,6 +49,7 @@ struct DevParams {
     int tc_tpc_min, tc_stages;        // tensor-core scorer: least tiles per block, K stages in shared memory
     int *fcnt, *fflag;                // fused scorer: per-unit counters of tiles in / of query rows merged ([2][units], contiguous)
     float *finz;                      // fused scorer: 1 / Z_r per unit and query row, [units][rows_pad]
+    int *qctrl;                       // work-queue counters of the one-block segmentation kernel, [4 + L * Bmax], zero between events
     float *logits;                    // narrow query blocks (rows_pad <= 16): scaled logits [units][T_cap][rows_pad], or null
     int *status;                      // [4]: code, unit, a, b
 };
@@ -169,6 +170,13 @@ __device__ __forceinline__ uint4 ld_stream16(const void *ptr)
     return v;
 }
 
+// 16-byte global store that is not kept in the caches (written once, read by a later kernel or never).
+__device__ __forceinline__ void st_stream16(void *ptr, uint4 v)
+{
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(ptr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+
 // Host-side launchers (one per translation unit).
 int tova_rows_block(int rows); // query rows handled per pass of the TOVA kernel (8..128)
 enum KernelId { kKernScore1 = 0, kKernScoreCombine, kKernScore2, kKernSegmentSelect, kKernGather, kKernTable, kKernUsage, kKernCount };
@@ -202,8 +210,10 @@ int launch_score_tova_fused(const DevParams &p, LaunchCtx &ctx);
 int launch_score_keydiff(const DevParams &p, LaunchCtx &ctx);
 int launch_segment_select(const DevParams &p, LaunchCtx &ctx);
 bool segment_cluster_supported(const DevParams &p);
+bool segment_moves_rows(const DevParams &p); // the segmentation launch also starts the paged compaction
 int launch_segment_select_cluster(const DevParams &p, LaunchCtx &ctx);
-int launch_gather(const DevParams &p, LaunchCtx &ctx);
+constexpr int kMoveRows = 512; // (token, head) rows of K and V per chunk of the paged compaction
+int launch_gather(const DevParams &p, LaunchCtx &ctx, bool queued); // queued: chunks below p.qctrl[1] are moved already
 int launch_smooth_usage(const DevParams &p, const float *src, float *dst, int k, LaunchCtx &ctx);
 
 } // namespace ams

@@ -12,17 +12,17 @@ constexpr int kRowsPerIter = kGatherThreads / 16;
 constexpr int kUnroll = 4;                   // K and V of 4 rows in flight per thread
 constexpr int kRowsPerBlock = kRowsPerIter * kUnroll;
 
-__device__ __forceinline__ void st_stream16(void *ptr, uint4 v)
-{
-    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(ptr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
-                 : "memory");
-}
-
 // Rows of one (layer, sequence) are numbered r = j * H + h, so that consecutive rows
 // are consecutive 256-byte pieces of the destination page.
-__global__ void __launch_bounds__(kGatherThreads) k_gather(DevParams p)
+// queued: the chunks (kMoveRows rows each, in (layer, sequence) order) below p.qctrl[1] were moved by the
+// segmentation kernel already.
+__global__ void __launch_bounds__(kGatherThreads) k_gather(DevParams p, int queued)
 {
     const int lb = blockIdx.y;
+    if (queued) {
+        const int chunks = (p.Tk * p.H + kMoveRows - 1) / kMoveRows;
+        if (lb * chunks + (int)(blockIdx.x * kRowsPerBlock) / kMoveRows < p.qctrl[1]) return;
+    }
     const int b = lb % p.B, l = lb / p.B;
     const int T = p.seq_lens[b];
     if (T <= p.Tk || T > p.T_cap) return;
@@ -68,17 +68,20 @@ __global__ void k_table_update(DevParams p)
     int *row = p.block_table + (size_t)b * p.bt_stride;
     for (int i = threadIdx.x; i < p.bt_stride; i += blockDim.x)
         row[i] = i < p.n_dst ? p.dst_pages[(size_t)b * p.n_dst + i] : -1;
+    if (b == 0) // work-queue counters of the segmentation kernel back to zero for the next event
+        for (int i = threadIdx.x; i < 4 + p.L * p.B; i += blockDim.x) p.qctrl[i] = 0;
     __syncthreads();
     if (threadIdx.x == 0) p.seq_lens[b] = p.Tk;
 }
 
 } // namespace
 
-int launch_gather(const DevParams &p, LaunchCtx &ctx)
+int launch_gather(const DevParams &p, LaunchCtx &ctx, bool queued)
 {
+    static_assert(kMoveRows % kRowsPerBlock == 0, "a block of the gather kernel lies inside one chunk");
     const int n_rows = p.Tk * p.H;
     dim3 grid((n_rows + kRowsPerBlock - 1) / kRowsPerBlock, p.L * p.B);
-    k_gather<<<grid, kGatherThreads, 0, ctx.s>>>(p);
+    k_gather<<<grid, kGatherThreads, 0, ctx.s>>>(p, queued ? 1 : 0);
     ctx.mark(kKernGather);
     k_table_update<<<p.B, 128, 0, ctx.s>>>(p);
     ctx.mark(kKernTable);

@@ -26,6 +26,7 @@ using namespace sel;
 namespace {
 
 constexpr int kXch = 8; // ring of exchange slots (>= 2)
+constexpr int kNT = 1024;
 
 // Dynamic shared memory of one block (byte offsets).
 struct SmemMap {
@@ -63,7 +64,7 @@ __host__ __device__ inline SmemMap smem_map(int tpc, int sc, int S, bool ema_on)
 // CS (blocks per cluster) is a template parameter so that every loop over the ranks of the cluster
 // unrolls into independent remote loads instead of a chain of dependent ones.
 template <int NT, int VPT, int CS>
-__global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, int cs_max)
+__device__ __forceinline__ void segment_unit(const DevParams &p, const int uid, const int cs_max)
 {
     constexpr int nt = NT, TPC = NT * VPT, cs = CS;
     extern __shared__ __align__(16) unsigned char dyn[];
@@ -73,7 +74,6 @@ __global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, i
     cg::cluster_group cluster = cg::this_cluster();
     const int tid = threadIdx.x, lane = tid & 31;
     const int rank = cs > 1 ? (int)cluster.block_rank() : 0;
-    const int uid = blockIdx.x / cs;
     const int h = uid % p.H, b = (uid / p.H) % p.B, l = uid / (p.H * p.B);
     const int T = p.seq_lens[b];
     // every exit below is taken by all blocks of the cluster together
@@ -781,6 +781,105 @@ __global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, i
 }
 
 template <int NT, int VPT, int CS>
+__global__ void __launch_bounds__(NT, 1) k_segment_select_cluster(DevParams p, int cs_max)
+{
+    segment_unit<NT, VPT, CS>(p, blockIdx.x / CS, cs_max);
+}
+
+// Work-queue form for sequences that fit one block: a persistent grid (one block per SM) takes the units
+// one by one.  Units rarely fill a whole number of waves, and their selection phases leave the memory
+// system idle: a block that finds no unit left starts on the paged compaction (the two display
+// equations of the paged-KV appendix: K_new[pi_new(b, j), h, :] <- K_old[pi_old(b, I_j), h, :], same
+// for V), chunk by chunk in (layer, sequence) order, for as long as other blocks are still selecting.
+// The gather kernel that follows moves the chunks that were not handed out (it has twice the threads
+// per SM, hence twice the bytes in flight, and is the faster mover once every SM is free).
+// ctrl: [0] next unit, [1] chunks handed out, [3] units finished, [4 + layer * B + b] heads of that
+// pair finished; the table-update kernel puts them back to zero.  A chunk is only ever handed out after
+// every unit has been handed out, so whoever it waits for is running; the wait is bounded all the same.
+constexpr uint32_t kDoneSpins = 1u << 22;
+
+template <int NT, int VPT>
+__global__ void __launch_bounds__(NT, 1) k_segment_select_move(DevParams p, int *ctrl)
+{
+    __shared__ int item_s;
+    const int tid = threadIdx.x;
+    const int units = p.L * p.B * p.H;
+    for (;;) {
+        __syncthreads(); // the previous unit's shared memory is no longer read
+        if (tid == 0) item_s = atomicAdd(&ctrl[0], 1);
+        __syncthreads();
+        const int uid = item_s;
+        if (uid >= units) break;
+        segment_unit<NT, VPT, 1>(p, uid, 1);
+        __syncthreads(); // every thread's writes of the unit (kept positions, credit) are issued
+        if (tid == 0) {
+            __threadfence();
+            atomicAdd(&ctrl[4 + uid / p.H], 1);
+            atomicAdd(&ctrl[3], 1);
+        }
+    }
+    const int rows_lb = p.Tk * p.H, chunks = (rows_lb + kMoveRows - 1) / kMoveRows, n_items = p.L * p.B * chunks;
+    for (;;) {
+        __syncthreads();
+        if (tid == 0) {
+            int it = n_items;
+            // once every unit is finished the rest is left to the gather kernel; the comparison and the
+            // claim are not atomic together, which at worst hands out one more chunk per block
+            if (*reinterpret_cast<const volatile int *>(ctrl + 3) < units) {
+                it = atomicAdd(&ctrl[1], 1);
+                if (it >= n_items) atomicSub(&ctrl[1], 1); // keep the count at the chunks really handed out
+            }
+            if (it < n_items) {
+                const volatile int *done = ctrl + 4 + it / chunks;
+                uint32_t spins = 0;
+                while (*done < p.H && ++spins < kDoneSpins) __nanosleep(128);
+                if (*done < p.H) { set_status(p.status, AMS_ERR_TIMEOUT, it, 0, 0); it = n_items; }
+                __threadfence();
+            }
+            item_s = it;
+        }
+        __syncthreads();
+        const int it = item_s;
+        if (it >= n_items) break;
+        const int lb = it / chunks, b = lb % p.B, l = lb / p.B;
+        const int T = p.seq_lens[b];
+        // sequences that were skipped or reported keep their rows
+        if (T <= p.Tk || T > p.T_cap) continue;
+        const int r_end = min(rows_lb, (it % chunks + 1) * kMoveRows);
+        const int *table = p.block_table + (size_t)b * p.bt_stride;
+        const int *dstp = p.dst_pages + (size_t)b * p.n_dst;
+        const int *keep_base = p.keep_idx + (size_t)lb * p.H * p.Tk;
+        const int l16 = tid & 15;
+        constexpr int kUnroll = 4, kRowsPerIter = NT / 16;
+        // rows are numbered r = j * H + h, so that consecutive rows are consecutive 256-byte pieces of the
+        // destination page
+        for (int r0 = (it % chunks) * kMoveRows + (tid >> 4); r0 < r_end; r0 += kRowsPerIter * kUnroll) {
+            uint4 kv[kUnroll], vv[kUnroll];
+            size_t doff[kUnroll];
+#pragma unroll
+            for (int i = 0; i < kUnroll; ++i) {
+                const int r = r0 + i * kRowsPerIter;
+                if (r < r_end) {
+                    const int j = r / p.H, h = r - j * p.H;
+                    const int pos = __ldcg(keep_base + (size_t)h * p.Tk + j);
+                    const size_t soff = row_offset(p, l, table[pos >> 4], pos & 15, h) + l16 * 8;
+                    doff[i] = row_offset(p, l, dstp[j >> 4], j & 15, h) + l16 * 8;
+                    kv[i] = ld_stream16(p.k_pages + soff);
+                    vv[i] = ld_stream16(p.v_pages + soff);
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < kUnroll; ++i) {
+                if (r0 + i * kRowsPerIter < r_end) {
+                    st_stream16(p.k_pages + doff[i], kv[i]);
+                    st_stream16(p.v_pages + doff[i], vv[i]);
+                }
+            }
+        }
+    }
+}
+
+template <int NT, int VPT, int CS>
 int launch_cfg(const DevParams &p, LaunchCtx &ctx, int cs_max, size_t smem)
 {
     static size_t configured = 0;
@@ -808,9 +907,44 @@ int launch_cfg(const DevParams &p, LaunchCtx &ctx, int cs_max, size_t smem)
     return AMS_OK;
 }
 
-constexpr int kNT = 1024;
-
 } // namespace
+
+// True when the work-queue kernel takes the call: every sequence fits one block.  It also moves part of the kept rows.
+static int sm_count()
+{
+    static int n_sm = 0;
+    if (!n_sm) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n_sm = 0;
+    }
+    return n_sm;
+}
+
+// With more units than SMs there is a last, partial wave to fill; with fewer the plain kernel is quicker.
+bool segment_moves_rows(const DevParams &p)
+{
+    return segment_cluster_supported(p) && p.T_cap <= kNT * 16 && sm_count() > 0 && p.L * p.B * p.H > sm_count();
+}
+
+template <int VPT>
+int launch_move(const DevParams &p, LaunchCtx &ctx, size_t smem)
+{
+    static size_t configured = 0;
+    const int n_sm = sm_count();
+    if (n_sm <= 0) return AMS_ERR_CUDA;
+    if (smem > configured) {
+        if (cudaFuncSetAttribute(k_segment_select_move<kNT, VPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return AMS_ERR_CUDA;
+        configured = smem;
+    }
+    const int units = p.L * p.B * p.H;
+    const int chunks = (p.Tk * p.H + kMoveRows - 1) / kMoveRows;
+    const int most = units > p.L * p.B * chunks ? units : p.L * p.B * chunks;
+    const int grid = most < n_sm ? most : n_sm;
+    k_segment_select_move<kNT, VPT><<<grid, kNT, smem, ctx.s>>>(p, p.qctrl);
+    ctx.mark(kKernSegmentSelect);
+    return cudaGetLastError() == cudaSuccess ? AMS_OK : AMS_ERR_CUDA;
+}
 
 // True when the on-chip kernel can take this call: the sequence capacity fits one cluster of
 // at most eight blocks and the segment tables fit beside the per-token arrays.
@@ -824,6 +958,11 @@ bool segment_cluster_supported(const DevParams &p)
 int launch_segment_select_cluster(const DevParams &p, LaunchCtx &ctx)
 {
     const bool ema_on = p.beta != 1.0f;
+    if (segment_moves_rows(p)) {
+        if (p.T_cap <= kNT * 4) return launch_move<4>(p, ctx, smem_map(kNT * 4, p.seg_cap, p.S, ema_on).total);
+        if (p.T_cap <= kNT * 8) return launch_move<8>(p, ctx, smem_map(kNT * 8, p.seg_cap, p.S, ema_on).total);
+        return launch_move<16>(p, ctx, smem_map(kNT * 16, p.seg_cap, p.S, ema_on).total);
+    }
     if (p.T_cap <= kNT * 4) return launch_cfg<kNT, 4, 1>(p, ctx, 1, smem_map(kNT * 4, p.seg_cap, p.S, ema_on).total);
     if (p.T_cap <= kNT * 8) return launch_cfg<kNT, 8, 1>(p, ctx, 1, smem_map(kNT * 8, p.seg_cap, p.S, ema_on).total);
     const int tpc = kNT * 16;
