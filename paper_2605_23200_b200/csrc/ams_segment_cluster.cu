@@ -850,29 +850,44 @@ __global__ void __launch_bounds__(NT, 1) k_segment_select_move(DevParams p, int 
         const int *dstp = p.dst_pages + (size_t)b * p.n_dst;
         const int *keep_base = p.keep_idx + (size_t)lb * p.H * p.Tk;
         const int l16 = tid & 15;
-        constexpr int kUnroll = 4, kRowsPerIter = NT / 16;
-        // rows are numbered r = j * H + h, so that consecutive rows are consecutive 256-byte pieces of the
-        // destination page
-        for (int r0 = (it % chunks) * kMoveRows + (tid >> 4); r0 < r_end; r0 += kRowsPerIter * kUnroll) {
+        constexpr int kUnroll = 4, kRowsPerIter = NT / 16, kStep = kRowsPerIter * kUnroll;
+        // Rows are numbered r = j * H + h, so that consecutive rows are consecutive 256-byte pieces of the
+        // destination page.  The source offsets of the next round (kept position, then its page: two
+        // dependent loads) are fetched while this round's rows are in flight.
+        auto source_of = [&](int r) -> size_t {
+            const int j = r / p.H, h = r - j * p.H;
+            const int pos = __ldcg(keep_base + (size_t)h * p.Tk + j);
+            return row_offset(p, l, table[pos >> 4], pos & 15, h) + l16 * 8;
+        };
+        const int r_first = (it % chunks) * kMoveRows + (tid >> 4);
+        size_t soff_next[kUnroll];
+#pragma unroll
+        for (int i = 0; i < kUnroll; ++i) {
+            const int r = r_first + i * kRowsPerIter;
+            soff_next[i] = r < r_end ? source_of(r) : 0;
+        }
+        for (int r0 = r_first; r0 < r_end; r0 += kStep) {
             uint4 kv[kUnroll], vv[kUnroll];
-            size_t doff[kUnroll];
+#pragma unroll
+            for (int i = 0; i < kUnroll; ++i) {
+                if (r0 + i * kRowsPerIter < r_end) {
+                    kv[i] = ld_stream16(p.k_pages + soff_next[i]);
+                    vv[i] = ld_stream16(p.v_pages + soff_next[i]);
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < kUnroll; ++i) {
+                const int r = r0 + kStep + i * kRowsPerIter;
+                soff_next[i] = r < r_end ? source_of(r) : 0;
+            }
 #pragma unroll
             for (int i = 0; i < kUnroll; ++i) {
                 const int r = r0 + i * kRowsPerIter;
                 if (r < r_end) {
                     const int j = r / p.H, h = r - j * p.H;
-                    const int pos = __ldcg(keep_base + (size_t)h * p.Tk + j);
-                    const size_t soff = row_offset(p, l, table[pos >> 4], pos & 15, h) + l16 * 8;
-                    doff[i] = row_offset(p, l, dstp[j >> 4], j & 15, h) + l16 * 8;
-                    kv[i] = ld_stream16(p.k_pages + soff);
-                    vv[i] = ld_stream16(p.v_pages + soff);
-                }
-            }
-#pragma unroll
-            for (int i = 0; i < kUnroll; ++i) {
-                if (r0 + i * kRowsPerIter < r_end) {
-                    st_stream16(p.k_pages + doff[i], kv[i]);
-                    st_stream16(p.v_pages + doff[i], vv[i]);
+                    const size_t doff = row_offset(p, l, dstp[j >> 4], j & 15, h) + l16 * 8;
+                    st_stream16(p.k_pages + doff, kv[i]);
+                    st_stream16(p.v_pages + doff, vv[i]);
                 }
             }
         }
