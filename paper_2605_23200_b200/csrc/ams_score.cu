@@ -340,23 +340,48 @@ __global__ void __launch_bounds__(kKdThreads) k_keydiff_score(DevParams p)
     for (int i = 0; i < 8; ++i) mu[i] = fin[lane * 8 + i];
     const float mu_norm = fin[kHeadDim];
     float *g_out = p.scores + (size_t)uid * p.T_cap;
-    const int n_iter = (t_end - t_begin + 15) >> 4;
+    // four tokens per thread and round: their loads are issued together, so that enough bytes are in flight
+    constexpr int kU = 4;
+    const int n_iter = (t_end - t_begin + 16 * kU - 1) / (16 * kU);
     for (int it = 0; it < n_iter; ++it) {
-        const int t = t_begin + it * 16 + r;
-        float dot = 0.0f, k2 = 0.0f;
-        if (t < t_end) {
-            const uint4 v = ld_stream16(p.k_pages + row_offset(p, l, table[t >> 4], t & 15, h) + lane * 8);
-            const float k[8] = {bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y),
-                                bf16_lo(v.z), bf16_hi(v.z), bf16_lo(v.w), bf16_hi(v.w)};
+        uint4 v[kU];
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+            const int t = t_begin + (it * kU + u) * 16 + r;
+            v[u] = make_uint4(0, 0, 0, 0);
+            if (t < t_end) v[u] = ld_stream16(p.k_pages + row_offset(p, l, table[t >> 4], t & 15, h) + lane * 8);
+        }
+        // a[2u] = this lane's part of k_t . mu, a[2u + 1] of |k_t|^2, for the four tokens u
+        float a[2 * kU];
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+            const float k[8] = {bf16_lo(v[u].x), bf16_hi(v[u].x), bf16_lo(v[u].y), bf16_hi(v[u].y),
+                                bf16_lo(v[u].z), bf16_hi(v[u].z), bf16_lo(v[u].w), bf16_hi(v[u].w)};
+            float dot = 0.0f, k2 = 0.0f;
 #pragma unroll
             for (int i = 0; i < 8; ++i) { dot = fmaf(k[i], mu[i], dot); k2 = fmaf(k[i], k[i], k2); }
+            a[2 * u] = dot; a[2 * u + 1] = k2;
         }
+        // sums over the 16 lanes of a token row, all eight values at once: at each step a lane hands half of
+        // its values to its partner and keeps the other half (9 shuffles instead of 32)
 #pragma unroll
-        for (int o = 1; o < 16; o <<= 1) {
-            dot += __shfl_xor_sync(0xffffffffu, dot, o);
-            k2 += __shfl_xor_sync(0xffffffffu, k2, o);
+        for (int o = 8, n = 2 * kU; o >= 2; o >>= 1, n >>= 1) {
+            const bool up = (lane & o) != 0;
+#pragma unroll
+            for (int i = 0; i < n / 2; ++i) {
+                const float send = up ? a[i] : a[i + n / 2];
+                const float keep = up ? a[i + n / 2] : a[i];
+                a[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+            }
         }
-        if (lane == 0 && t < t_end) g_out[t] = -dot / fmaxf(sqrtf(k2) * mu_norm, 1e-30f);
+        a[0] += __shfl_xor_sync(0xffffffffu, a[0], 1);
+        // lane holds value index 4 * bit3 + 2 * bit2 + bit1: even = dot of token (index / 2), odd = its |k|^2
+        const float other = __shfl_xor_sync(0xffffffffu, a[0], 2);
+        if ((lane & 3) == 0) {
+            const int u = lane >> 2;
+            const int t = t_begin + (it * kU + u) * 16 + r;
+            if (t < t_end) g_out[t] = -a[0] / fmaxf(sqrtf(other) * mu_norm, 1e-30f);
+        }
     }
 }
 

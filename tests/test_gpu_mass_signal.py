@@ -138,7 +138,11 @@ def test_keydiff_ranking_with_window_attention_mass(k):
     cache0 = inputs.make_cache(wl0, DEV)
     comp0 = binding.AmsCompressor(binding.config_for(wl0), DEV)
     dbg0 = gpu_event(comp0, cache0, inputs.alloc_dst_pages(cache0))
-    assert torch.equal(dbg0.scores, dbg0.usage) and torch.equal(dbg0.scores, dbg.scores)
+    assert torch.equal(dbg0.scores, dbg0.usage)
+    for b in range(wl.batch):                       # positions beyond a sequence's length are never written
+        T = int(snap.lens[b])
+        if T > wl.budget:
+            assert torch.equal(dbg0.scores[:, b, :, :T], dbg.scores[:, b, :, :T])
 
 
 def test_mass_signal_argument_errors():

@@ -143,7 +143,9 @@ def _check_scorer(wl, rtol=1e-3, atol=0.0, sample_units=None):
             want = oracle.score_keydiff(snap.k, l, h, snap.table[b], T)
         assert_scores_close(got[l, b, h, :T], want, rtol, atol)
         _, _, m_want = oracle.mass(want, wl.eps)
-        assert_scores_close(mass[l, b, h, :T], m_want, rtol, 1e-3 * wl.eps)
+        # an absolute slack on a score is that slack over the sum of the weights on its mass (Eq. 1)
+        sum_w = float(np.maximum(want.astype(np.float64), 0.0).sum() + wl.eps * T)
+        assert_scores_close(mass[l, b, h, :T], m_want, rtol, 1e-3 * wl.eps + atol / sum_w)
     # selection on the library's own scores is exactly what the oracle selects on those scores
     compare_event(snap, cache, comp, dbg, dst, credit0, got, units=sample_units)
     return comp, cache
