@@ -64,6 +64,10 @@ EXT_CASES = [
                   n_last=0, q_min=0, ema_beta=1.0)),                                           # global top-k over 4 blocks
     ("spike", dict(seq_len_min=50000, seq_len_max=50000, budget=6000, batch=1, n_layers=1, n_kv_heads=2, n_q_heads=8)),
     ("ties", dict(seq_len_min=3000, seq_len_max=3000, budget=700, l_min=1, l_max=5, n_segments=64, q_min=2)),  # many tiny segments
+    # more units than SMs (work-queue form of the segmentation kernel, row moves split with the gather kernel):
+    # ragged with skipped sequences, and a budget that is not a multiple of the page size
+    ("lognormal", dict(n_layers=4, batch=9, seq_len_min=500, seq_len_max=2600, budget=1203, n_last=5)),
+    ("ties", dict(n_layers=5, batch=4, seq_len_min=4000, seq_len_max=9000, budget=2048, ema_beta=1.0, n_segments=12)),
 ]
 
 
