@@ -177,6 +177,27 @@ __device__ __forceinline__ void st_stream16(void *ptr, uint4 v)
                  : "memory");
 }
 
+// A kernel launched with launch_after may start (prologue, loads that depend on nothing the previous kernel of
+// the stream writes) while that kernel's last blocks are still running; it calls wait_for_previous_kernel() before
+// it first touches anything the previous kernel wrote, or anything that kernel still reads and this one writes.
+__device__ __forceinline__ void wait_for_previous_kernel() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_after(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // Host-side launchers (one per translation unit).
 int tova_rows_block(int rows); // query rows handled per pass of the TOVA kernel (8..128)
 enum KernelId { kKernScore1 = 0, kKernScoreCombine, kKernScore2, kKernSegmentSelect, kKernGather, kKernTable, kKernUsage, kKernCount };

@@ -18,6 +18,7 @@ constexpr int kRowsPerBlock = kRowsPerIter * kUnroll;
 // segmentation kernel already.
 __global__ void __launch_bounds__(kGatherThreads) k_gather(DevParams p, int queued)
 {
+    wait_for_previous_kernel(); // kept positions and the count of chunks already moved
     const int lb = blockIdx.y;
     if (queued) {
         const int chunks = (p.Tk * p.H + kMoveRows - 1) / kMoveRows;
@@ -62,6 +63,7 @@ __global__ void __launch_bounds__(kGatherThreads) k_gather(DevParams p, int queu
 // every kernel that reads the old table.
 __global__ void k_table_update(DevParams p)
 {
+    wait_for_previous_kernel(); // the gather kernel reads the table this kernel rewrites
     const int b = blockIdx.x;
     const int T = p.seq_lens[b];
     if (T <= p.Tk || T > p.T_cap) return;
@@ -81,9 +83,9 @@ int launch_gather(const DevParams &p, LaunchCtx &ctx, bool queued)
     static_assert(kMoveRows % kRowsPerBlock == 0, "a block of the gather kernel lies inside one chunk");
     const int n_rows = p.Tk * p.H;
     dim3 grid((n_rows + kRowsPerBlock - 1) / kRowsPerBlock, p.L * p.B);
-    k_gather<<<grid, kGatherThreads, 0, ctx.s>>>(p, queued ? 1 : 0);
+    if (launch_after(k_gather, grid, dim3(kGatherThreads), 0, ctx.s, p, queued ? 1 : 0) != cudaSuccess) return AMS_ERR_CUDA;
     ctx.mark(kKernGather);
-    k_table_update<<<p.B, 128, 0, ctx.s>>>(p);
+    if (launch_after(k_table_update, dim3((unsigned)p.B), dim3(128), 0, ctx.s, p) != cudaSuccess) return AMS_ERR_CUDA;
     ctx.mark(kKernTable);
     return cudaGetLastError() == cudaSuccess ? AMS_OK : AMS_ERR_CUDA;
 }

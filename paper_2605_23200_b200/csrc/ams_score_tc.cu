@@ -258,7 +258,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
                     }
                 } else {
                     // merge the statistics the blocks of the first pass left for this unit, in block
-                    // order: b_r = M_r + log2 Z_r per row, and the window maximum 1 / min_r Z_r
+                    // order: b_r = M_r + log2 Z_r per row, and the window maximum 1 / min_r Z_r.
+                    // This pass is launched so that its blocks may start while the last blocks of the first
+                    // pass are still running (its loads and MMAs depend on nothing the first pass writes);
+                    // only here, before the statistics are read, must the first pass be complete.
+                    if (seg == 0) wait_for_previous_kernel();
                     const int nt_u = prefix[s.b + 1] - prefix[s.b];
                     const long long ustart = g - s.tile0;
                     const int n_parts = (int)((ustart + nt_u - 1) / tpc) - (int)(ustart / tpc) + 1;
@@ -489,7 +493,7 @@ int launch_score_tova_tc(const DevParams &p, LaunchCtx &ctx)
     const int grid = groups * p.H;
     k_tova_tc<1><<<grid, kTcThreads, smem, ctx.s>>>(p, k_map, q_map);
     ctx.mark(kKernScore1);
-    k_tova_tc<2><<<grid, kTcThreads, smem, ctx.s>>>(p, k_map, q_map);
+    if (launch_after(k_tova_tc<2>, dim3((unsigned)grid), dim3(kTcThreads), smem, ctx.s, p, k_map, q_map) != cudaSuccess) return AMS_ERR_CUDA;
     ctx.mark(kKernScore2);
     return cudaGetLastError() == cudaSuccess ? AMS_OK : AMS_ERR_CUDA;
 }

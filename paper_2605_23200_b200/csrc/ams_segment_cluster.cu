@@ -804,6 +804,7 @@ __global__ void __launch_bounds__(NT, 1) k_segment_select_move(DevParams p, int 
     __shared__ int item_s;
     const int tid = threadIdx.x;
     const int units = p.L * p.B * p.H;
+    wait_for_previous_kernel(); // the scores
     for (;;) {
         __syncthreads(); // the previous unit's shared memory is no longer read
         if (tid == 0) item_s = atomicAdd(&ctrl[0], 1);
@@ -956,9 +957,9 @@ int launch_move(const DevParams &p, LaunchCtx &ctx, size_t smem)
     const int chunks = (p.Tk * p.H + kMoveRows - 1) / kMoveRows;
     const int most = units > p.L * p.B * chunks ? units : p.L * p.B * chunks;
     const int grid = most < n_sm ? most : n_sm;
-    k_segment_select_move<kNT, VPT><<<grid, kNT, smem, ctx.s>>>(p, p.qctrl);
+    if (launch_after(k_segment_select_move<kNT, VPT>, dim3((unsigned)grid), dim3(kNT), smem, ctx.s, p, p.qctrl) != cudaSuccess) return AMS_ERR_CUDA;
     ctx.mark(kKernSegmentSelect);
-    return cudaGetLastError() == cudaSuccess ? AMS_OK : AMS_ERR_CUDA;
+    return AMS_OK;
 }
 
 // True when the on-chip kernel can take this call: the sequence capacity fits one cluster of
