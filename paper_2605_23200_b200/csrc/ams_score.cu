@@ -59,6 +59,7 @@ __global__ void __launch_bounds__(kTovaThreads) k_tova(DevParams p)
 {
     __shared__ __align__(16) __nv_bfloat16 Qs[NTB > 1 ? NTB * 8 * kQPitch : 8];
     __shared__ float red[4][NTB * 8][2];
+    if (PHASE == 2) wait_for_previous_kernel(); // merged statistics
     const int uid = blockIdx.y, slice = blockIdx.x;
     const int h = uid % p.H, b = (uid / p.H) % p.B, l = uid / (p.H * p.B);
     const int T = p.seq_lens[b];
@@ -214,6 +215,7 @@ __global__ void __launch_bounds__(kTovaThreads) k_tova(DevParams p)
 __global__ void __launch_bounds__(128) k_tova_combine(DevParams p)
 {
     __shared__ u64 scratch[40];
+    wait_for_previous_kernel(); // the slices' statistics
     const int uid = blockIdx.x;
     const int b = (uid / p.H) % p.B;
     const int T = p.seq_lens[b];
@@ -245,6 +247,7 @@ template <int RP>
 __global__ void __launch_bounds__(256) k_tova_usage_from_logits(DevParams p)
 {
     __shared__ float bs[RP + 1];
+    wait_for_previous_kernel(); // merged statistics (and, through that kernel, the logits)
     const int uid = blockIdx.x;
     const int b = (uid / p.H) % p.B;
     const int T = p.seq_lens[b];
@@ -304,6 +307,7 @@ __global__ void __launch_bounds__(kKdThreads) k_keydiff_sum(DevParams p)
 __global__ void __launch_bounds__(kHeadDim) k_keydiff_combine(DevParams p)
 {
     __shared__ float sq[kHeadDim];
+    wait_for_previous_kernel(); // the slices' sums
     const int uid = blockIdx.x;
     const int b = (uid / p.H) % p.B;
     const int T = p.seq_lens[b];
@@ -325,6 +329,7 @@ __global__ void __launch_bounds__(kHeadDim) k_keydiff_combine(DevParams p)
 
 __global__ void __launch_bounds__(kKdThreads) k_keydiff_score(DevParams p)
 {
+    wait_for_previous_kernel(); // the mean key
     const int uid = blockIdx.y, slice = blockIdx.x;
     const int h = uid % p.H, b = (uid / p.H) % p.B, l = uid / (p.H * p.B);
     const int T = p.seq_lens[b];
@@ -391,13 +396,13 @@ void launch_tova_ntb(const DevParams &p, LaunchCtx &ctx)
     const dim3 grid(p.n_slices, p.L * p.B * p.H);
     k_tova<NTB, 1><<<grid, kTovaThreads, 0, ctx.s>>>(p);
     ctx.mark(kKernScore1);
-    k_tova_combine<<<p.L * p.B * p.H, 128, 0, ctx.s>>>(p);
+    launch_after(k_tova_combine, dim3((unsigned)(p.L * p.B * p.H)), dim3(128), 0, ctx.s, p);
     ctx.mark(kKernScoreCombine);
     if (NTB <= 2 && p.logits && p.rows_pad == NTB * 8) {
         const dim3 g2(p.L * p.B * p.H, (p.T_cap + 255) / 256);
-        k_tova_usage_from_logits<NTB * 8><<<g2, 256, 0, ctx.s>>>(p);
+        launch_after(k_tova_usage_from_logits<NTB * 8>, g2, dim3(256), 0, ctx.s, p);
     } else {
-        k_tova<NTB, 2><<<grid, kTovaThreads, 0, ctx.s>>>(p);
+        launch_after(k_tova<NTB, 2>, grid, dim3(kTovaThreads), 0, ctx.s, p);
     }
     ctx.mark(kKernScore2);
 }
@@ -430,9 +435,9 @@ int launch_score_keydiff(const DevParams &p, LaunchCtx &ctx)
     const dim3 grid(p.n_slices, p.L * p.B * p.H);
     k_keydiff_sum<<<grid, kKdThreads, 0, ctx.s>>>(p);
     ctx.mark(kKernScore1);
-    k_keydiff_combine<<<p.L * p.B * p.H, kHeadDim, 0, ctx.s>>>(p);
+    launch_after(k_keydiff_combine, dim3((unsigned)(p.L * p.B * p.H)), dim3(kHeadDim), 0, ctx.s, p);
     ctx.mark(kKernScoreCombine);
-    k_keydiff_score<<<grid, kKdThreads, 0, ctx.s>>>(p);
+    launch_after(k_keydiff_score, grid, dim3(kKdThreads), 0, ctx.s, p);
     ctx.mark(kKernScore2);
     return cudaGetLastError() == cudaSuccess ? AMS_OK : AMS_ERR_CUDA;
 }
