@@ -12,9 +12,10 @@ Prints ONE JSON line (rank 0).  `value` = whole-job steps/s with the cache resid
 HBM, timed with CUDA events on the launching stream.  `e2e` = the same through the
 C ABI with the step's inputs (observation queries, block table, lengths,
 replacement pages) copied from pinned host memory and its results (block table,
-lengths, device status) read back and waited for inside the timed region; the upload
-of the next step's inputs overlaps the current step's kernels (two input buffer
-sets), as a serving loop would do; the paged K/V pool is the persistent device
+lengths) read back and checked inside the timed region; the upload of the next
+step's inputs and the read-back of the previous step's results overlap the current
+step's kernels (three buffer sets, at most two steps in flight), as a serving loop
+would do; the paged K/V pool is the persistent device
 state the step operates on and is not copied.
 """
 from __future__ import annotations
@@ -222,31 +223,47 @@ def run_ours(args, rank, world, local_rank):
     # Two sets of device input buffers: while step i computes, the inputs of step i + 1 are uploaded on a second
     # stream (what a serving loop does); every step still uploads all its inputs from pinned host memory, and
     # its results (block table, lengths, device status) are read back and waited for before the next launch.
-    sets = [(q, cache.block_table, cache.seq_lens, dst),
-            (None if q is None else torch.empty_like(q), torch.empty_like(cache.block_table), torch.empty_like(cache.seq_lens),
-             torch.empty_like(dst))]
+    NB = 3  # buffer sets: one being uploaded, one computing, one being read back
+    sets = [(q, cache.block_table, cache.seq_lens, dst)] + [
+        (None if q is None else torch.empty_like(q), torch.empty_like(cache.block_table), torch.empty_like(cache.seq_lens),
+         torch.empty_like(dst)) for _ in range(NB - 1)]
     copy_stream = torch.cuda.Stream(dev)
-    uploaded = [torch.cuda.Event(), torch.cuda.Event()]
+    uploaded = [torch.cuda.Event() for _ in range(NB)]
 
     def upload(i):
-        qi, ti, li, di = sets[i & 1]
+        qi, ti, li, di = sets[i % NB]
         with torch.cuda.stream(copy_stream):
             if host_q is not None:
                 qi.copy_(host_q, non_blocking=True)
             ti.copy_(host_table, non_blocking=True)
             li.copy_(host_lens, non_blocking=True)
             di.copy_(host_dst, non_blocking=True)
-            uploaded[i & 1].record(copy_stream)
+            uploaded[i % NB].record(copy_stream)
+
+    read_stream = torch.cuda.Stream(dev)
+    computed = [torch.cuda.Event() for _ in range(NB)]
+    read_back = [torch.cuda.Event() for _ in range(NB)]
+    outs = [(out_table, out_lens)] + [(torch.empty_like(out_table).pin_memory(), torch.empty_like(out_lens).pin_memory())
+                                      for _ in range(NB - 1)]
+
+    def check(i):                           # results of step i: wait for their read-back and look at them
+        read_back[i % NB].synchronize()
+        assert int(outs[i % NB][1][0]) == wl.budget
 
     def e2e_step(i):
-        qi, ti, li, di = sets[i & 1]
-        upload(i + 1)                       # overlaps this step's kernels; its buffers were released by the wait below
-        stream.wait_event(uploaded[i & 1])
+        qi, ti, li, di = sets[i % NB]
+        if i >= 2:
+            check(i - 2)                    # also releases the buffer set that upload(i + 1) is about to fill
+        upload(i + 1)                       # overlaps the kernels of steps i - 1 and i
+        stream.wait_event(uploaded[i % NB])
         comp.ema_state.zero_()
         comp.compress(cache.k_pages, cache.v_pages, ti, li, qi, wl.budget, wl.n_segments, wl.scorer_id, di)
-        out_table.copy_(ti, non_blocking=True)
-        out_lens.copy_(li, non_blocking=True)
-        comp.status()  # reads the device status word and synchronises the stream
+        computed[i % NB].record(stream)
+        with torch.cuda.stream(read_stream):  # block table and lengths of this step back to pinned host memory
+            read_stream.wait_event(computed[i % NB])
+            outs[i % NB][0].copy_(ti, non_blocking=True)
+            outs[i % NB][1].copy_(li, non_blocking=True)
+            read_back[i % NB].record(read_stream)
 
     n_e2e = min(args.steps, 50)
     e2e_ms = None
@@ -255,13 +272,18 @@ def run_ours(args, rank, world, local_rank):
         upload(0)
         for i in range(3):
             e2e_step(i)
+        check(1)
+        check(2)
+        comp.status()
         barrier()
         t0 = time.perf_counter()
         for i in range(3, 3 + n_e2e):
             e2e_step(i)
+        check(1 + n_e2e)
+        check(2 + n_e2e)
+        comp.status()  # device status word of the whole run; synchronises the stream
         torch.cuda.synchronize(dev)
         e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3, dev)
-        assert int(out_lens[0]) == wl.budget
 
     k_read, moved = algorithmic_bytes(wl, lens0.cpu().numpy())
     peak, peak_kind = _peaks()
@@ -294,7 +316,7 @@ def run_ours(args, rank, world, local_rank):
                              "frac is of the measured copy bandwidth"},
         "e2e": None if e2e_ms is None else {"value": world * n_e2e / (e2e_ms / 1e3), "unit": UNIT,
                                             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e,
-                                            "note": "uploads of step i+1 overlap the kernels of step i (two input buffer sets)"},
+                                            "note": "uploads of step i+1 and the read-back of step i-1 overlap the kernels of step i (three buffer sets, three streams, at most two steps in flight); every step uploads all its inputs and its block table and lengths are read back and checked"},
         "clocks": clocks,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
