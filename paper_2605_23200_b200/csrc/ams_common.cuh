@@ -47,6 +47,7 @@ struct DevParams {
     float *fin;                       // per unit finals
     int slice_len, n_slices, rows_pad;
     int tc_tpc_min, tc_stages;        // tensor-core scorer: least tiles per block, K stages in shared memory
+    int tc_hpb;                       // tensor-core scorer: KV heads a block takes one after the other (set by its launcher)
     int *fcnt, *fflag;                // fused scorer: per-unit counters of tiles in / of query rows merged ([2][units], contiguous)
     float *finz;                      // fused scorer: 1 / Z_r per unit and query row, [units][rows_pad]
     int *qctrl;                       // work-queue counters of the one-block segmentation kernel, [4 + L * Bmax], zero between events

@@ -1,8 +1,8 @@
 // TOVA-style scorer for wide observation windows (rows = G * W >= 64) on the sm_100a
 // tensor path: tcgen05.mma with TMEM accumulators, operands staged by TMA.
 //
-// Work is the concatenation of all units' 128-token tiles; block c of a persistent grid
-// takes the contiguous tile range [c * tpc, (c + 1) * tpc).  Inside a block:
+// Work is the concatenation of all units' 128-token tiles; a group of blocks of a persistent grid
+// takes the contiguous tile range [g * tpc, (g + 1) * tpc) for all KV heads (one or more heads per block).  Inside a block:
 //   warp 0      TMA producer: query block of the current unit, then one 32 KB K tile per
 //               stage (eight 16-token pages, one 4 KB copy each, 128-byte swizzle);
 //   warps 1, 3  MMA issuers (one lane each, one per pair of consumer warpgroups, tiles in
@@ -123,8 +123,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    const int my_h = blockIdx.x % p.H, my_group = blockIdx.x / p.H;
-    tc_partition(p, gridDim.x / p.H, prefix, &sh.tiles_lh, &sh.n_tiles, &sh.tpc);
+    // A group of H / tc_hpb blocks walks one range of token tiles; block j of the group takes KV heads
+    // j, j + H / tc_hpb, ... one after the other over that range (tc_hpb > 1 where H alone does not divide
+    // the SM count well: 148 SMs and 8 heads give 18 groups of 8 blocks, or 37 groups of 4 with two heads each).
+    const int hpb = p.tc_hpb, my_hs = p.H / hpb;
+    const int my_h0 = blockIdx.x % my_hs, my_group = blockIdx.x / my_hs;
+    tc_partition(p, gridDim.x / my_hs, prefix, &sh.tiles_lh, &sh.n_tiles, &sh.tpc);
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)), "r"(512) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -136,6 +140,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
     const int tiles_lh = sh.tiles_lh, tpc = sh.tpc;
     const long long g_begin = (long long)my_group * tpc;
     const long long g_end = (g_begin + tpc < sh.n_tiles) ? g_begin + tpc : sh.n_tiles;
+    const long long g_span = g_end - g_begin; // the loops below run over hpb * g_span tiles: head after head
     if (PHASE == 1 && blockIdx.x == 0 && tid == 0) {
         for (int b = 0; b < p.B; ++b) {
             const int T = p.seq_lens[b];
@@ -149,7 +154,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
             // ------------------------------------------------------------ TMA producer
             int kit = 0, seg = 0, issued = 0;
             bool ok = true;
-            for (long long g = g_begin; g < g_end && ok;) {
+            for (long long gv = 0; gv < g_span * hpb && ok;) {
+                const int my_h = my_h0 + (int)(gv / g_span) * my_hs;
+                const long long g = g_begin + gv % g_span;
                 const Segment s = decode_segment(p, prefix, tiles_lh, tpc, g, g_end, my_h);
                 ok = mbar_wait(smem_u32(&sh.qempty), (uint32_t)((seg & 1) ^ 1), abort_flag);
                 if (!ok) break;
@@ -179,7 +186,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
                     }
                     issued = kit + 1;
                 }
-                g += s.n;
+                gv += s.n;
                 ++seg;
             }
             if (!ok) { // drain: wait (bounded) for the copies that were issued and never consumed
@@ -197,7 +204,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
                 const int wg = warp >> 1; // issuer 0 feeds consumer pair 0 (even tiles), issuer 1 pair 1
                 int kit = 0, seg = 0, wsit = 0; // wsit: accumulator slots handed to the warpgroup so far
                 bool ok = true;
-                for (long long g = g_begin; g < g_end && ok;) {
+                for (long long gv = 0; gv < g_span * hpb && ok;) {
+                const int my_h = my_h0 + (int)(gv / g_span) * my_hs;
+                const long long g = g_begin + gv % g_span;
                     const Segment s = decode_segment(p, prefix, tiles_lh, tpc, g, g_end, my_h);
                     ok = mbar_wait(smem_u32(&sh.qfull), (uint32_t)(seg & 1), abort_flag);
                     for (int i = 0; i < s.n && ok; ++i, ++kit) {
@@ -223,7 +232,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
                         if (ok) tc_commit(smem_u32(&sh.kempty[st]));
                     }
                     if (ok) tc_commit(smem_u32(&sh.qempty));
-                    g += s.n;
+                    gv += s.n;
                     ++seg;
                 }
                 // all tensor work issued by this thread has finished before TMEM is released
@@ -242,7 +251,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
             bool ok = true;
             // a thread whose wait ran out keeps walking the segments without touching the pipeline, so that
             // the consumers' named barriers stay matched
-            for (long long g = g_begin; g < g_end;) {
+            for (long long gv = 0; gv < g_span * hpb;) {
+                const int my_h = my_h0 + (int)(gv / g_span) * my_hs;
+                const long long g = g_begin + gv % g_span;
                 const Segment s = decode_segment(p, prefix, tiles_lh, tpc, g, g_end, my_h);
                 const int T = s.T;
                 float m[4], z[4];
@@ -418,7 +429,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
                     }
                     asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory"); // the buffer is free again
                 }
-                g += s.n;
+                gv += s.n;
                 ++seg;
             }
         }
@@ -441,8 +452,9 @@ size_t tova_tc_smem_bytes(const DevParams &p)
            (size_t)3 * (p.rows_pad / 128) * 128 * 8 + 256;
 }
 
-int launch_score_tova_tc(const DevParams &p, LaunchCtx &ctx)
+int launch_score_tova_tc(const DevParams &p_in, LaunchCtx &ctx)
 {
+    DevParams p = p_in; // the launcher fills in how the heads are spread over the blocks
     // With two MMA issuers taking tiles in turn, an even ring depth gives every stage to one issuer, which
     // then sees all phases of the stage's barrier in order (a parity wait must not skip a phase).
     if (p.tc_stages < 2 || (p.tc_stages & 1)) return AMS_ERR_UNSUPPORTED;
@@ -488,9 +500,18 @@ int launch_score_tova_tc(const DevParams &p, LaunchCtx &ctx)
     }
     const long long cap_tiles = (long long)p.L * p.B * ((p.T_cap + kTileTokens - 1) / kTileTokens); // per head
     long long want = (cap_tiles + p.tc_tpc_min - 1) / p.tc_tpc_min;
-    const int max_groups = n_sm / p.H;
+    // heads per block: the divisor of H that fills most SMs (the smallest one on a tie)
+    int hpb = 1;
+    for (int d = 1, best = 0; d <= p.H; ++d) {
+        if (p.H % d) continue;
+        const int blocks = n_sm / (p.H / d) * (p.H / d);
+        if (blocks > best) { best = blocks; hpb = d; }
+    }
+    const int nh = p.H / hpb;
+    const int max_groups = n_sm / nh;
     const int groups = (int)(want < max_groups ? (want < 1 ? 1 : want) : max_groups);
-    const int grid = groups * p.H;
+    const int grid = groups * nh;
+    p.tc_hpb = hpb;
     k_tova_tc<1><<<grid, kTcThreads, smem, ctx.s>>>(p, k_map, q_map);
     ctx.mark(kKernScore1);
     if (launch_after(k_tova_tc<2>, dim3((unsigned)grid), dim3(kTcThreads), smem, ctx.s, p, k_map, q_map) != cudaSuccess) return AMS_ERR_CUDA;
