@@ -147,7 +147,11 @@ int ams_init_state(const ams_config *cfg, void *ema_state, void *workspace, size
  * zero-padded average over k neighbouring positions: u'_t = (sum of u_j, |j - t| <= k/2, j inside
  * the sequence, added left to right in fp32) / k.
  *  dbg              : optional views, or NULL.
- * Calls on the same handle share the workspace and must not overlap on the GPU. */
+ * Calls on the same handle share the workspace and must not overlap on the GPU.  The call allocates
+ * nothing and never synchronises; after one direct call (which sets kernel attributes) it can be captured
+ * into a CUDA graph.  Its kernels follow one another on `stream` as dependent launches (a kernel may start
+ * while its predecessor's last blocks run and waits before touching that kernel's output); work enqueued
+ * on `stream` before or after the call is ordered as usual. */
 int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages, int32_t *block_table,
                  int32_t block_table_stride, int32_t *seq_lens, int32_t batch, const void *obs_queries,
                  int32_t window, void *ema_state, int32_t budget, int32_t n_segments, int32_t scorer_id,
