@@ -36,7 +36,8 @@ def build(force: bool = False) -> str:
 class _Params(ctypes.Structure):
     _fields_ = [("n_segments", ctypes.c_int32), ("l_min", ctypes.c_int32), ("l_max", ctypes.c_int32),
                 ("q_min", ctypes.c_int32), ("n_sink", ctypes.c_int32), ("n_last", ctypes.c_int32),
-                ("ema_lambda", ctypes.c_float), ("ema_beta", ctypes.c_float), ("eps", ctypes.c_float)]
+                ("ema_lambda", ctypes.c_float), ("ema_beta", ctypes.c_float), ("eps", ctypes.c_float),
+                ("fixed_segments", ctypes.c_int32), ("uniform_quotas", ctypes.c_int32)]
 
 
 @dataclass
@@ -52,10 +53,12 @@ class Params:
     ema_lambda: float = 0.9
     ema_beta: float = 0.9
     eps: float = 1e-8
+    fixed_segments: bool = False    # ablation: equal-length instead of equal-mass segments
+    uniform_quotas: bool = False    # ablation: budget shared by segment length instead of mass
 
     def c(self) -> _Params:
         return _Params(self.n_segments, self.l_min, self.l_max, self.q_min, self.n_sink, self.n_last,
-                       self.ema_lambda, self.ema_beta, self.eps)
+                       self.ema_lambda, self.ema_beta, self.eps, int(self.fixed_segments), int(self.uniform_quotas))
 
     def max_segments(self, T: int) -> int:
         cap = self.n_segments

@@ -48,6 +48,8 @@ typedef struct {
     float ema_lambda;   /* credit decay                                          */
     float ema_beta;     /* mixing weight of the current mass; 1 = credit unused  */
     float eps;          /* Eq. 1 epsilon                                         */
+    int32_t fixed_segments; /* ablation "fixed-length segments": cuts at k T / S   */
+    int32_t uniform_quotas; /* ablation "w/o mass-weighted quotas": share by length */
 } orc_params;
 
 /* ------------------------------------------------------------------------- */
@@ -497,13 +499,35 @@ int32_t orc_select_unit(const float *u, const float *g, float *credit, int32_t T
     orc_mass(u, T, prm->eps, A, &SA, m);
     orc_history_mass(A, SA, m, credit, T, prm->ema_lambda, prm->ema_beta, Hm);
     orc_prefix(Hm, T, C);
-    const int32_t n_raw = orc_cuts(C, T, prm->n_segments, raw);
+    int32_t n_raw;
+    if (prm->fixed_segments) {
+        /* component ablation of the paper: S segments of equal length instead of equal mass,
+         * boundary k at floor(k T / S); merge and split then act as usual */
+        n_raw = 0;
+        raw[n_raw++] = 0;
+        for (int k = 1; k < prm->n_segments; ++k) {
+            const int32_t cut = (int32_t)(((int64_t)k * T) / prm->n_segments);
+            if (cut > raw[n_raw - 1] && cut < T) raw[n_raw++] = cut;
+        }
+        raw[n_raw++] = T;
+    } else {
+        n_raw = orc_cuts(C, T, prm->n_segments, raw);
+    }
     const int32_t nb = orc_merge_split(raw, n_raw, prm->l_min, prm->l_max, bounds, cap + 1);
     if (nb < 2) { ret = -3; goto done; }
     const int32_t n_seg = nb - 1;
     int32_t ns, nl;
     orc_must_keep(T, Tk, prm->n_sink, prm->n_last, &ns, &nl);
-    orc_quotas(C, bounds, n_seg, prm->q_min, Tk - ns - nl, q);
+    if (prm->uniform_quotas) {
+        /* component ablation of the paper: the budget is shared by segment length, not by mass:
+         * the quota routine sees a "mass" of one per token */
+        uint64_t *ones = (uint64_t *)malloc(sizeof(uint64_t) * (size_t)T);
+        for (int t = 0; t < T; ++t) ones[t] = (uint64_t)t + 1;
+        orc_quotas(ones, bounds, n_seg, prm->q_min, Tk - ns - nl, q);
+        free(ones);
+    } else {
+        orc_quotas(C, bounds, n_seg, prm->q_min, Tk - ns - nl, q);
+    }
     const int32_t nbf = orc_select(g, T, bounds, q, n_seg, ns, nl, Tk, keep_idx);
     if (nbf < 0) { ret = -4; goto done; }
     if (prm->ema_beta != 1.0f) {

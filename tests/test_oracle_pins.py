@@ -538,3 +538,37 @@ def test_smoothing_changes_the_mass_only_and_decoupled_signals_split_roles():
     for unit in both:
         assert (both[unit].bounds == only_u[unit].bounds).all() and (both[unit].quotas == only_u[unit].quotas).all()
         assert (both[unit].mass == only_u[unit].mass).all()
+
+
+# ----------------------------------------------------------------------------- component ablations
+
+def test_ablation_fixed_length_segments_and_length_proportional_quotas():
+    """The two component ablations of the paper's ablation table: segments of equal length, and a
+    budget shared by segment length instead of mass."""
+    rng = np.random.default_rng(77)
+    T, Tk, S = 1200, 300, 10
+    u = np.exp(2.0 * rng.standard_normal(T)).astype(np.float32)
+    base = dict(n_segments=S, l_min=1, l_max=0, q_min=1, n_sink=0, n_last=0, ema_beta=1.0)
+    # fixed-length: S divides T, so every boundary is k T / S whatever the mass looks like
+    r = oracle.select_unit(u, u, None, Tk, Params(fixed_segments=True, **base))
+    assert r.bounds.tolist() == [k * T // S for k in range(S + 1)]
+    r2 = oracle.select_unit(np.roll(u, 123), None, None, Tk, Params(fixed_segments=True, **base))
+    assert r2.bounds.tolist() == r.bounds.tolist() and r2.quotas.tolist() != r.quotas.tolist()  # quotas still follow the mass
+    # S does not divide T: floor(k T / S), then the usual merge of short pieces
+    r3 = oracle.select_unit(u[:1003], None, None, Tk, Params(fixed_segments=True, **base))
+    assert r3.bounds.tolist() == [k * 1003 // S for k in range(S + 1)]
+    r4 = oracle.select_unit(u[:1003], None, None, Tk, Params(fixed_segments=True, **{**base, "l_min": 150}))
+    assert r4.bounds[0] == 0 and r4.bounds[-1] == 1003 and (np.diff(r4.bounds) >= 150).all()
+    # length-proportional quotas: equal lengths -> equal quotas, however skewed the mass is
+    r5 = oracle.select_unit(u, None, None, Tk, Params(fixed_segments=True, uniform_quotas=True, **base))
+    assert r5.quotas.tolist() == [Tk // S] * S
+    # with mass-quantile segments of different lengths: quotas follow the lengths within one token and sum to the budget
+    r6 = oracle.select_unit(u, None, None, Tk, Params(uniform_quotas=True, **base))
+    L = np.diff(r6.bounds)
+    assert r6.quotas.sum() == Tk and (np.abs(r6.quotas - Tk * L / T) <= 1.0 + 1e-9).all()
+    assert (r6.bounds == oracle.select_unit(u, None, None, Tk, Params(**base)).bounds).all()   # segments unchanged
+    # inside a segment the pick is still the top-q of the scores
+    for i in range(r6.n_seg):
+        a, b = r6.bounds[i], r6.bounds[i + 1]
+        top = sorted(range(a, b), key=lambda t: (-u[t], t))[: r6.quotas[i]]
+        assert set(top) <= set(r6.keep_idx.tolist())
