@@ -92,6 +92,11 @@ typedef struct {
                                                 step 1, optional smoothing); 1 = none         */
     int32_t decoupled;                       /* 1: reserve room for a mass signal that differs
                                                 from the base scores (see ams_compress)       */
+    int32_t fixed_segments;                  /* 1: component ablation "fixed-length segments":
+                                                cut k at floor(k seq_len / S) instead of at the
+                                                mass quantile; merge and split as usual       */
+    int32_t uniform_quotas;                  /* 1: component ablation "w/o mass-weighted quotas":
+                                                the budget is shared by segment length        */
 } ams_config;
 
 /* Optional device outputs for inspection and tests; any member may be NULL.
@@ -110,7 +115,7 @@ typedef struct {
 
 /* Paper defaults: segment mass 0.1 (n_segments = 10 is passed per call), lengths
  * 16 / 256, q_min 1, lambda = beta = 0.9, 4 sinks; n_last 16, eps 1e-8; pool_kernel 1 (no
- * smoothing), decoupled 0.  Geometry and capacities are zeroed and must be filled by the caller. */
+ * smoothing), decoupled 0, both ablation switches 0.  Geometry and capacities are zeroed and must be filled by the caller. */
 void ams_config_default(ams_config *cfg);
 
 /* Sizes of the caller-allocated device buffers; 0 if the configuration is invalid. */

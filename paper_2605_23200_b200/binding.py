@@ -33,7 +33,8 @@ class AmsConfig(ctypes.Structure):
                 ("n_layers", "n_q_heads", "n_kv_heads", "head_dim", "page_size", "max_batch", "max_seq_len",
                  "max_window", "max_budget", "max_segments", "l_min", "l_max", "q_min", "n_sink", "n_last")] + \
                [("ema_lambda", ctypes.c_float), ("ema_beta", ctypes.c_float), ("eps", ctypes.c_float),
-                ("causal_window", ctypes.c_int32), ("pool_kernel", ctypes.c_int32), ("decoupled", ctypes.c_int32)]
+                ("causal_window", ctypes.c_int32), ("pool_kernel", ctypes.c_int32), ("decoupled", ctypes.c_int32),
+                ("fixed_segments", ctypes.c_int32), ("uniform_quotas", ctypes.c_int32)]
 
 
 class AmsDebugViews(ctypes.Structure):
@@ -245,4 +246,5 @@ def config_for(wl, **kw) -> AmsConfig:
                           max_budget=wl.budget, max_segments=max(wl.n_segments, 1), l_min=wl.l_min, l_max=wl.l_max,
                           q_min=wl.q_min, n_sink=wl.n_sink, n_last=wl.n_last, ema_lambda=wl.ema_lambda,
                           ema_beta=wl.ema_beta, eps=wl.eps, pool_kernel=wl.pool_kernel, decoupled=int(wl.decoupled),
+                          fixed_segments=int(wl.fixed_segments), uniform_quotas=int(wl.uniform_quotas),
                           **kw)

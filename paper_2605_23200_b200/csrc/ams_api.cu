@@ -28,6 +28,7 @@ static bool config_ok(const ams_config *c, int *why)
     if (!(c->eps > 0.0f) || !(c->eps < 1e30f)) return false;
     if (c->pool_kernel < 1 || c->pool_kernel > 63 || !(c->pool_kernel & 1)) return false;
     if (c->decoupled != 0 && c->decoupled != 1) return false;
+    if ((c->fixed_segments != 0 && c->fixed_segments != 1) || (c->uniform_quotas != 0 && c->uniform_quotas != 1)) return false;
     *why = AMS_ERR_UNSUPPORTED;
     if (c->head_dim != kHeadDim || c->page_size != kPage) return false;
     if (c->n_q_heads % c->n_kv_heads) return false;
@@ -144,6 +145,8 @@ void ams_config_default(ams_config *cfg)
     cfg->causal_window = 1;
     cfg->pool_kernel = 1;
     cfg->decoupled = 0;
+    cfg->fixed_segments = 0;
+    cfg->uniform_quotas = 0;
 }
 
 size_t ams_ema_state_bytes(const ams_config *cfg)
@@ -230,6 +233,7 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
     p.T_cap = y.T_cap; p.seg_cap = y.seg_cap; p.Tk = budget; p.S = n_segments; p.n_dst = (budget + kPage - 1) / kPage;
     p.l_min = c.l_min; p.l_max = c.l_max; p.q_min = c.q_min; p.n_sink = c.n_sink; p.n_last = c.n_last;
     p.causal = c.causal_window ? 1 : 0;
+    p.fixed_seg = c.fixed_segments; p.uniform_q = c.uniform_quotas;
     p.lambda = c.ema_lambda; p.beta = c.ema_beta; p.eps = c.eps;
     p.k_pages = (__nv_bfloat16 *)k_pages; p.v_pages = (__nv_bfloat16 *)v_pages; p.num_pages = num_pages;
     p.block_table = block_table; p.bt_stride = block_table_stride; p.seq_lens = seq_lens;

@@ -22,6 +22,7 @@ struct DevParams {
     int L, B, Bmax, H, G, W, rows;    // rows = G * W query rows per KV head
     int T_cap, seg_cap, Tk, S, n_dst; // n_dst = ceil(Tk / 16)
     int l_min, l_max, q_min, n_sink, n_last, causal;
+    int fixed_seg, uniform_q;         // component ablations: equal-length segments, quotas by segment length
     float lambda, beta, eps;
     // caller buffers
     __nv_bfloat16 *k_pages, *v_pages;

@@ -136,6 +136,10 @@ __global__ void __launch_bounds__(1024) k_segment_select(DevParams p)
         }
     }
     __syncthreads();
+    if (p.fixed_seg) { // component ablation: boundary k at floor(k T / S) whatever the mass
+        for (int k = tid + 1; k < p.S; k += nt) raw[k] = (int)(((long long)k * T) / p.S);
+        __syncthreads();
+    }
 
     // ---- merge short raw segments forward, fold a short tail left, count split pieces
     if (tid == 0) {
@@ -175,10 +179,11 @@ __global__ void __launch_bounds__(1024) k_segment_select(DevParams p)
     const int ns = max(0, min(p.n_sink, min(p.Tk, T)));
     const int nl = max(0, min(p.n_last, min(p.Tk - ns, T - ns)));
     const int Bq = p.Tk - ns - nl;
+    const u64 SHq = p.uniform_q ? (u64)T : SH; // total of what the quotas are proportional to
     long long smin = 0;
     for (int i = tid; i < n_seg; i += nt) {
         const int a = bounds[i], e = bounds[i + 1];
-        Ms[i] = Cb[e - 1] - (a > 0 ? Cb[a - 1] : 0ull);
+        Ms[i] = p.uniform_q ? (u64)(e - a) : Cb[e - 1] - (a > 0 ? Cb[a - 1] : 0ull); // ablation: share by length
         smin += max(0, min(p.q_min, e - a));
     }
     smin = block_sum_i64(smin, sm.scratch);
@@ -187,7 +192,7 @@ __global__ void __launch_bounds__(1024) k_segment_select(DevParams p)
     for (int i = tid; i < n_seg; i += nt) {
         const int L = bounds[i + 1] - bounds[i];
         long long qi = max(0, min(p.q_min, L));
-        if (Trem >= 0) qi += (long long)((2ull * (u64)Trem * Ms[i] + SH) / (2ull * SH));
+        if (Trem >= 0) qi += (long long)((2ull * (u64)Trem * Ms[i] + SHq) / (2ull * SHq));
         if (qi > L) qi = L;
         quota[i] = (int)qi;
         sq += qi;

@@ -284,7 +284,9 @@ __device__ __forceinline__ void segment_unit(const DevParams &p, const int uid, 
         }
         return lo;
     };
-    if (my0 < n_loc) {
+    if (p.fixed_seg) { // component ablation: boundary k at floor(k T / S) whatever the mass (every block, own copy)
+        for (int k = tid + 1; k < p.S; k += nt) raw[k] = (int)(((long long)k * T) / p.S);
+    } else if (my0 < n_loc) {
         int kprev = quantile(exc);
         const int klast = quantile(exc + tt);
         if (klast != kprev) {
@@ -391,9 +393,10 @@ __device__ __forceinline__ void segment_unit(const DevParams &p, const int uid, 
     const int ns = max(0, min(p.n_sink, min(p.Tk, T)));
     const int nl = max(0, min(p.n_last, min(p.Tk - ns, T - ns)));
     const int Bq = p.Tk - ns - nl;
+    const u64 SHq = p.uniform_q ? (u64)T : SH; // total of what the quotas are proportional to
     long long smin = 0;
     for (int i = tid; i < n_seg; i += nt) {
-        Ms[i] = Cend[i] - (i > 0 ? Cend[i - 1] : 0ull);
+        Ms[i] = p.uniform_q ? (u64)(bounds[i + 1] - bounds[i]) : Cend[i] - (i > 0 ? Cend[i - 1] : 0ull); // ablation: share by length
         smin += max(0, min(p.q_min, bounds[i + 1] - bounds[i]));
     }
     smin = block_sum_i64(smin, sm.scratch);
@@ -402,7 +405,7 @@ __device__ __forceinline__ void segment_unit(const DevParams &p, const int uid, 
     for (int i = tid; i < n_seg; i += nt) {
         const int L = bounds[i + 1] - bounds[i];
         long long qi = max(0, min(p.q_min, L));
-        if (Trem >= 0) qi += (long long)((2ull * (u64)Trem * Ms[i] + SH) / (2ull * SH));
+        if (Trem >= 0) qi += (long long)((2ull * (u64)Trem * Ms[i] + SHq) / (2ull * SHq));
         if (qi > L) qi = L;
         quota[i] = (int)qi;
         sq += qi;

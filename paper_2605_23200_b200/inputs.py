@@ -62,6 +62,8 @@ class Workload:
     resident_layers: int = 0  # 0 = all layers resident
     pool_kernel: int = 1      # width of the average pooling of the usage scores (1 = none)
     decoupled: bool = False   # key-only base scores with the window attention as mass signal
+    fixed_segments: bool = False  # ablation: equal-length instead of equal-mass segments
+    uniform_quotas: bool = False  # ablation: budget shared by segment length instead of mass
 
     @property
     def group(self) -> int:

@@ -11,7 +11,7 @@ from paper_2605_23200_b200 import binding, inputs
 
 def params_of(wl) -> oracle.Params:
     return oracle.Params(wl.n_segments, wl.l_min, wl.l_max, wl.q_min, wl.n_sink, wl.n_last, wl.ema_lambda,
-                         wl.ema_beta, wl.eps)
+                         wl.ema_beta, wl.eps, wl.fixed_segments, wl.uniform_quotas)
 
 
 class HostSnapshot:
