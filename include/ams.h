@@ -111,6 +111,13 @@ typedef struct {
     int32_t *seg_bounds; /* [L][batch][H][C+1] boundaries a_0 = 0 < ... < a_n = seq_len     */
     int32_t *quotas;     /* [L][batch][H][C]                                                 */
     int32_t *keep_idx;   /* [L][batch][H][budget] kept positions, ascending                 */
+    /* Diagnostic of the paper's mechanistic-diagnostics appendix: retained-set IoU between the previous
+     * event and this one.  prev_kept (input, DEVICE int32 [batch], may be NULL) gives, per sequence, how
+     * many tokens at the front of the cache are the retained set of the previous event (the previous
+     * budget; 0 for a sequence never compressed).  With both pointers set, retained_iou receives
+     * |R_prev & R_now| / |R_prev | R_now| per unit, R_now being this event's kept tokens. */
+    const int32_t *prev_kept;
+    float *retained_iou; /* [L][batch][H] */
 } ams_debug_views;
 
 /* Paper defaults: segment mass 0.1 (n_segments = 10 is passed per call), lengths

@@ -275,6 +275,17 @@ def gather_unit(k_pages, v_pages, layer, h, table_row, dst_row, keep_idx):
                           ctypes.c_int32(len(keep_idx)))
 
 
+def retained_iou(keep_idx, prev_kept, budget):
+    """Retained-set IoU between two consecutive compression events of one (layer, sequence, KV
+    head) (mechanistic-diagnostics appendix): the previous event left its `prev_kept` retained
+    tokens at positions [0, prev_kept) of the cache; `keep_idx` are the positions this event keeps.
+    IoU = |R_prev & R_now| / |R_prev | R_now| on token identities; float32."""
+    prev = set(range(int(prev_kept)))
+    now = set(int(t) for t in keep_idx[:budget])
+    union = len(prev | now)
+    return np.float32(0.0) if union == 0 else np.float32(len(prev & now)) / np.float32(union)
+
+
 # --------------------------------------------------------------------------- whole event
 
 SCORER_TOVA, SCORER_KEYDIFF, SCORER_EXTERNAL = 0, 1, 2

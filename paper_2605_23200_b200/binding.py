@@ -38,7 +38,8 @@ class AmsConfig(ctypes.Structure):
 
 
 class AmsDebugViews(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_void_p) for n in ("scores", "usage", "mass", "n_segments", "seg_bounds", "quotas", "keep_idx")]
+    _fields_ = [(n, ctypes.c_void_p) for n in ("scores", "usage", "mass", "n_segments", "seg_bounds", "quotas", "keep_idx", "prev_kept",
+                                                "retained_iou")]
 
 
 _lib = None
@@ -124,11 +125,13 @@ class DebugViews:
     seg_bounds: torch.Tensor
     quotas: torch.Tensor
     keep_idx: torch.Tensor
+    prev_kept: torch.Tensor | None = None       # input: int32 [batch], previous event's retained count per sequence
+    retained_iou: torch.Tensor | None = None    # output: float32 [L][batch][H]
 
     def c(self) -> AmsDebugViews:
-        return AmsDebugViews(*(t.data_ptr() for t in
+        return AmsDebugViews(*(None if t is None else t.data_ptr() for t in
                                (self.scores, self.usage, self.mass, self.n_segments, self.seg_bounds, self.quotas,
-                                self.keep_idx)))
+                                self.keep_idx, self.prev_kept, self.retained_iou)))
 
 
 class AmsCompressor:

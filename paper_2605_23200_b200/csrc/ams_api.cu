@@ -301,6 +301,7 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
         if (dbg->quotas && e == cudaSuccess) e = cudaMemcpyAsync(dbg->quotas, p.quotas, U * (size_t)p.seg_cap * 4, cudaMemcpyDeviceToDevice, s);
         if (dbg->keep_idx && e == cudaSuccess) e = cudaMemcpyAsync(dbg->keep_idx, p.keep_idx, U * (size_t)p.Tk * 4, cudaMemcpyDeviceToDevice, s);
         if (e != cudaSuccess) rc = AMS_ERR_CUDA;
+        if (rc == AMS_OK && dbg->prev_kept && dbg->retained_iou) rc = launch_retained_iou(p, dbg->prev_kept, dbg->retained_iou, ctx);
     }
     if (rc == AMS_OK) rc = launch_gather(p, ctx, queued);
     st->last_launches = ctx.launches;

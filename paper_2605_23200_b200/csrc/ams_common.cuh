@@ -238,5 +238,6 @@ int launch_segment_select_cluster(const DevParams &p, LaunchCtx &ctx);
 constexpr int kMoveRows = 512; // (token, head) rows of K and V per chunk of the paged compaction
 int launch_gather(const DevParams &p, LaunchCtx &ctx, bool queued); // queued: chunks below p.qctrl[1] are moved already
 int launch_smooth_usage(const DevParams &p, const float *src, float *dst, int k, LaunchCtx &ctx);
+int launch_retained_iou(const DevParams &p, const int *prev_kept, float *out, LaunchCtx &ctx); // before the lengths are rewritten
 
 } // namespace ams

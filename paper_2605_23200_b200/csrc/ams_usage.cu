@@ -34,7 +34,36 @@ __global__ void __launch_bounds__(kSmoothThreads) k_smooth_usage(DevParams p, co
     dst[(size_t)uid * p.T_cap + t] = out;
 }
 
+// Retained-set IoU between the previous event and this one (mechanistic-diagnostics appendix of the
+// paper), one thread per unit: the previous retained set occupies positions [0, prev) of the cache, the
+// kept positions are ascending, so the intersection is the number of kept positions below prev.
+__global__ void __launch_bounds__(128) k_retained_iou(DevParams p, const int *prev_kept, float *out)
+{
+    const int uid = blockIdx.x * 128 + threadIdx.x;
+    if (uid >= p.L * p.B * p.H) return;
+    const int b = (uid / p.H) % p.B;
+    const int T = p.seq_lens[b];
+    if (T <= p.Tk || T > p.T_cap) return;
+    const int prev = max(0, min(prev_kept[b], T));
+    const int *keep = p.keep_idx + (size_t)uid * p.Tk;
+    int lo = 0, hi = p.Tk; // first kept position that is not below prev
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (keep[mid] < prev) lo = mid + 1; else hi = mid;
+    }
+    const int both = lo, either = prev + p.Tk - both;
+    out[uid] = either > 0 ? __fdiv_rn((float)both, (float)either) : 0.0f;
+}
+
 } // namespace
+
+int launch_retained_iou(const DevParams &p, const int *prev_kept, float *out, LaunchCtx &ctx)
+{
+    const int units = p.L * p.B * p.H;
+    k_retained_iou<<<(units + 127) / 128, 128, 0, ctx.s>>>(p, prev_kept, out);
+    ++ctx.launches;
+    return cudaGetLastError() == cudaSuccess ? AMS_OK : AMS_ERR_CUDA;
+}
 
 int launch_smooth_usage(const DevParams &p, const float *src, float *dst, int k, LaunchCtx &ctx)
 {

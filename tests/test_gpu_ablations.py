@@ -44,3 +44,38 @@ def test_ablation_switches_bit_exact(kw):
         for (l, b, h), r in res.items():
             T = int(snap.lens[b])
             assert r.bounds.tolist() == sorted(set(k * T // wl.n_segments for k in range(wl.n_segments + 1)))
+
+
+def test_retained_set_iou_between_consecutive_events():
+    """Diagnostic of the mechanistic-diagnostics appendix: after an event the retained tokens sit at the
+    front of the cache; the next event's IoU with them follows from its kept positions alone."""
+    import oracle
+    wl = inputs.CONFIGS[2].scaled(resident_layers=0, n_layers=2, batch=3, seq_len_min=700, seq_len_max=1300, budget=256,
+                                  append_per_step=96, steps=3)
+    cache = inputs.make_cache(wl, DEV)
+    comp = binding.AmsCompressor(binding.config_for(wl), DEV)
+    prev = torch.zeros(wl.batch, dtype=torch.int32, device=DEV)
+    for step in range(wl.steps):
+        dst_np = inputs.alloc_dst_pages(cache)
+        lens = cache.seq_lens.cpu().numpy().copy()
+        dbg = comp.make_debug_views(wl.batch, wl.budget)
+        dbg.prev_kept = prev
+        dbg.retained_iou = torch.full((wl.n_layers, wl.batch, wl.n_kv_heads), -1.0, device=DEV)
+        comp.compress(cache.k_pages, cache.v_pages, cache.block_table, cache.seq_lens, cache.obs_queries, wl.budget,
+                      wl.n_segments, wl.scorer_id, torch.from_numpy(dst_np).to(DEV), dbg=dbg)
+        comp.status()
+        keep = dbg.keep_idx.cpu().numpy()
+        got = dbg.retained_iou.cpu().numpy()
+        for l in range(wl.n_layers):
+            for b in range(wl.batch):
+                for h in range(wl.n_kv_heads):
+                    if lens[b] <= wl.budget:
+                        assert got[l, b, h] == -1.0                      # skipped sequences are left untouched
+                    else:
+                        assert got[l, b, h] == oracle.retained_iou(keep[l, b, h], int(prev[b]), wl.budget), (step, l, b, h)
+        if step > 0:
+            assert (got[got >= 0] > 0.3).all() and (got <= 1.0).all()    # most of a retained set survives 96 new tokens
+        prev = torch.from_numpy(np.where(lens > wl.budget, wl.budget, 0).astype(np.int32)).to(DEV)
+        inputs.after_compress(cache, dst_np)
+        if step + 1 < wl.steps:
+            inputs.append_tokens(cache, wl.append_per_step)

@@ -572,3 +572,13 @@ def test_ablation_fixed_length_segments_and_length_proportional_quotas():
         a, b = r6.bounds[i], r6.bounds[i + 1]
         top = sorted(range(a, b), key=lambda t: (-u[t], t))[: r6.quotas[i]]
         assert set(top) <= set(r6.keep_idx.tolist())
+
+
+def test_retained_iou_closed_forms():
+    Tk = 8
+    assert oracle.retained_iou(np.arange(Tk), Tk, Tk) == np.float32(1.0)                 # the same set twice
+    assert oracle.retained_iou(np.arange(Tk, 2 * Tk), Tk, Tk) == np.float32(0.0)         # only new tokens kept
+    keep = np.array([0, 2, 4, 6, 8, 9, 10, 11])                                          # four old, four new
+    assert oracle.retained_iou(keep, Tk, Tk) == np.float32(4) / np.float32(12)
+    assert oracle.retained_iou(keep, 0, Tk) == np.float32(0.0)                           # no previous event
+    assert oracle.retained_iou(keep, 5, Tk) == np.float32(3) / np.float32(10)            # a smaller previous budget
