@@ -26,9 +26,15 @@
  * off; lambda = 0 => credit equals mass; gather equals dense indexing; TOVA
  * with one query row => library softmax; KeyDiff => library cosine similarity;
  * usage smoothing => library zero-padded average pooling and a hand-computed case.
- * Parity unpinned (invariants only): merge direction and the order of merge vs
- * split; the choice of "roughly equal" split sizes; rounding rule of the quota
- * share; the padding value of the causal observation window when W > 1.
+ * EMA weights (beta on the current mass, 1 - beta on the normalised credit) and
+ * the must-keep order (suffix gives way before the sinks) against exact rationals
+ * and hand-worked cases; quota rounding (halves up) and the visiting order of the
+ * adjustment step against hand-worked cases; the reciprocal normalisation against
+ * exact integer division.
+ * Parity unpinned (invariants and hand-made examples of this reading only, the
+ * paper fixes neither): merge direction and the order of merge vs split; the
+ * choice of "roughly equal" split sizes; the padding value of the causal
+ * observation window when W > 1.
  */
 #include <float.h>
 #include <math.h>
