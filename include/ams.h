@@ -38,14 +38,18 @@
  * on fixed-point images of the mass, so they do not depend on summation order.
  *
  * Scorer selection is automatic (query rows per KV head >= 64: tensor-core path, otherwise the
- * mma.sync path).  Setting the environment variable AMS_FUSED_SCORER=1 selects an experimental
- * scorer that reads K once (query rows padded to 128, sequences up to 148 tiles of 128 tokens);
- * it is slower than the default at the sizes measured so far.
+ * mma.sync path) and depends on the arguments only: no environment variable changes what runs.
  *
  * Errors: every function returns AMS_OK (0) or a negative code.  Calls are
- * asynchronous on `stream`; conditions found on the device (a sequence longer
- * than max_seq_len, a window longer than a sequence, a bounded wait that ran out)
- * skip the affected work and are reported by ams_get_status.
+ * asynchronous on `stream`; conditions found on the device are reported by
+ * ams_get_status.  The first kernel of an event checks every sequence: one longer
+ * than max_seq_len (AMS_ERR_CAPACITY), one shorter than the observation window, or
+ * one whose block-table row or replacement pages name a page outside [0, num_pages)
+ * (AMS_ERR_INVALID_ARG, detail = sequence, index in the row, page id) is skipped
+ * entirely: its pages, table row, length and credit stay as they were.  A bounded
+ * wait that ran out is AMS_ERR_TIMEOUT.  The library serves any number of devices
+ * per process (launch state is kept per device); a handle belongs to the device that
+ * was current when it was created.
  */
 #ifndef AMS_H_
 #define AMS_H_
@@ -175,6 +179,12 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
  * unit index and two values describing it. */
 int ams_get_status(ams_state *st, void *stream, int32_t *detail);
 
+/* Failure-handling check without a failure: enqueues a one-thread kernel that waits on a barrier
+ * nobody arrives at, gives up after `polls` polls (1 .. 2^20) and records AMS_ERR_TIMEOUT in the
+ * handle's status word, the way the bounded waits inside the tensor-core scorer do when they run
+ * out.  The next ams_get_status returns that code; nothing else is touched. */
+int ams_debug_expire_wait(ams_state *st, uint32_t polls, void *stream);
+
 /* Number of kernels the last ams_compress on this handle launched. */
 int32_t ams_last_launch_count(const ams_state *st);
 
@@ -183,7 +193,7 @@ int32_t ams_last_launch_count(const ams_state *st);
  * device memory is allocated).  ams_get_kernel_times waits for the last call's final
  * event and writes AMS_KERNEL_SLOTS durations in milliseconds, one per kernel slot
  * named by ams_kernel_name (a slot launched more than once holds the sum). */
-#define AMS_KERNEL_SLOTS 7
+#define AMS_KERNEL_SLOTS 10
 int ams_set_profiling(ams_state *st, int enable);
 int ams_get_kernel_times(ams_state *st, float *ms);
 const char *ams_kernel_name(int32_t idx);
@@ -196,7 +206,7 @@ const char *ams_kernel_name(int32_t idx);
  * must-keep, backfill) on caller-supplied scores and writes the kept positions; there is
  * no EMA credit (the mass is that of the given scores alone), no K/V movement, no handle
  * and no workspace argument.  The scratch is a fixed device array inside the library
- * (about 2.6 MB, held by every GPU that loads the library until the process exits).
+ * (about 2.4 MB, held by every GPU that loads the library until the process exits).
  *   scores   : DEVICE fp32 [n_units][score_stride], score_stride a multiple of 16, >= seq_len
  *   keep_idx : DEVICE int32 [n_units][budget], ascending positions
  *   cfg      : only l_min, l_max, q_min, n_sink, n_last and eps are read
@@ -209,6 +219,13 @@ const char *ams_kernel_name(int32_t idx);
  * graph replayed concurrently) race on it.  Asynchronous on `stream`. */
 int ams_select_static(const ams_config *cfg, const float *scores, int32_t score_stride, int32_t n_units,
                       int32_t seq_len, int32_t budget, int32_t n_segments, int32_t *keep_idx, void *stream);
+
+/* Status of the ams_select_static calls on the current device: synchronises `stream`, returns and
+ * clears the first condition their kernels found on the device (AMS_ERR_CAPACITY: more segments
+ * than the fixed array holds; AMS_ERR_INTERNAL: a kept-count check failed), AMS_OK otherwise.  A unit
+ * that reported leaves its keep_idx row as the caller passed it.  detail[0..3] (host, may be NULL)
+ * as in ams_get_status.  Allocates nothing (the paper has no counterpart). */
+int ams_select_static_status(int32_t *detail, void *stream);
 
 /* Releases the host handle only. */
 int ams_free(ams_state *st);

@@ -24,8 +24,9 @@ AMS_SCORER_TOVA, AMS_SCORER_KEYDIFF, AMS_SCORER_EXTERNAL = 0, 1, 2
 
 EXPORTS = ["ams_config_default", "ams_ema_state_bytes", "ams_workspace_bytes", "ams_segment_capacity",
            "ams_init_state", "ams_compress", "ams_get_status", "ams_last_launch_count", "ams_free",
-           "ams_strerror", "ams_set_profiling", "ams_get_kernel_times", "ams_kernel_name", "ams_select_static"]
-KERNEL_SLOTS = 7
+           "ams_strerror", "ams_set_profiling", "ams_get_kernel_times", "ams_kernel_name", "ams_select_static",
+           "ams_select_static_status", "ams_debug_expire_wait"]
+KERNEL_SLOTS = 10
 
 
 class AmsConfig(ctypes.Structure):
@@ -84,6 +85,10 @@ def lib() -> ctypes.CDLL:
                                         ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p,
                                         ctypes.c_void_p]
         L.ams_select_static.restype = ctypes.c_int
+        L.ams_select_static_status.argtypes = [ctypes.POINTER(ctypes.c_int32), ctypes.c_void_p]
+        L.ams_select_static_status.restype = ctypes.c_int
+        L.ams_debug_expire_wait.argtypes = [ctypes.c_void_p, ctypes.c_uint32, ctypes.c_void_p]
+        L.ams_debug_expire_wait.restype = ctypes.c_int
         L.ams_strerror.argtypes = [ctypes.c_int]
         L.ams_strerror.restype = ctypes.c_char_p
         _lib = L
@@ -198,6 +203,13 @@ class AmsCompressor:
             raise AmsError(rc, "device status", list(detail))
         return rc, list(detail)
 
+    def expire_wait(self, polls: int = 1000, stream: torch.cuda.Stream | None = None) -> None:
+        """Failure-handling check: a bounded device wait that runs out after `polls` polls."""
+        s = stream or torch.cuda.current_stream(self.device)
+        rc = lib().ams_debug_expire_wait(self._h, polls, ctypes.c_void_p(s.cuda_stream))
+        if rc != AMS_OK:
+            raise AmsError(rc, "ams_debug_expire_wait")
+
     def set_profiling(self, enable: bool) -> None:
         rc = lib().ams_set_profiling(self._h, 1 if enable else 0)
         if rc != AMS_OK:
@@ -240,6 +252,14 @@ def select_static(cfg: AmsConfig, scores: torch.Tensor, seq_len: int, budget: in
                                  n_segments, _ptr(keep_idx), ctypes.c_void_p(s.cuda_stream))
     if rc != AMS_OK:
         raise AmsError(rc, "ams_select_static")
+
+
+def select_static_status(stream: torch.cuda.Stream | None = None, device="cuda:0"):
+    """(code, detail) of the allocation-free entry point's device status on the current device; clears it."""
+    s = stream or torch.cuda.current_stream(torch.device(device))
+    detail = (ctypes.c_int32 * 4)()
+    rc = lib().ams_select_static_status(detail, ctypes.c_void_p(s.cuda_stream))
+    return rc, list(detail)
 
 
 def config_for(wl, **kw) -> AmsConfig:

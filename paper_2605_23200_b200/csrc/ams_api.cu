@@ -8,7 +8,7 @@
 namespace ams {
 
 struct Layout {
-    size_t status, scores, usage, logits, qctrl, cbuf, flags, n_seg, seg_bounds, quotas, keep_idx, part, fin, ctrl, finz, total;
+    size_t status, eff_lens, seq_bad, scores, usage, logits, qctrl, cbuf, flags, n_seg, raw_cuts, seg_bounds, quotas, keep_idx, part, fin, total;
     int units, T_cap, seg_cap, n_slices, slice_len, rows_pad_cap;
 };
 
@@ -80,18 +80,18 @@ static Layout make_layout(const ams_config *c)
     if (tc_parts > y.n_slices) y.n_slices = tc_parts;
     const int rows_cap = (c->n_q_heads / c->n_kv_heads) * (c->max_window > 0 ? c->max_window : 1);
     y.rows_pad_cap = rows_padded(rows_cap);
-    // single-pass scorer (query rows padded to 128, sequences of at most 148 tiles): one partial per 128-token tile
-    const int tiles_cap = (y.T_cap + 127) / 128;
-    if (rows_cap >= 64 && y.rows_pad_cap >= 128 && tiles_cap <= 148 && tiles_cap > y.n_slices) y.n_slices = tiles_cap;
     const size_t U = (size_t)y.units, T = (size_t)y.T_cap;
     size_t off = 0;
     y.status = off;     off = align_up(off + 64, 256);
+    y.eff_lens = off;   off = align_up(off + (size_t)c->max_batch * 4, 256);
+    y.seq_bad = off;    off = align_up(off + (size_t)c->max_batch * 4, 256);
     y.scores = off;     off = align_up(off + U * T * 4, 256);
     // second per-token array: the usage when it is smoothed or comes from another scorer than the base scores
     y.usage = off;      off = align_up(off + ((c->pool_kernel > 1 || c->decoupled) ? U * T * 4 : 0), 256);
     y.cbuf = off;       off = align_up(off + U * T * 8, 256);
     y.flags = off;      off = align_up(off + U * T, 256);
     y.n_seg = off;      off = align_up(off + U * 4, 256);
+    y.raw_cuts = off;   off = align_up(off + U * (size_t)(c->max_segments + 1) * 4, 256);
     y.seg_bounds = off; off = align_up(off + U * (size_t)(y.seg_cap + 1) * 4, 256);
     y.quotas = off;     off = align_up(off + U * (size_t)y.seg_cap * 4, 256);
     y.keep_idx = off;   off = align_up(off + U * (size_t)c->max_budget * 4, 256);
@@ -102,9 +102,7 @@ static Layout make_layout(const ams_config *c)
     // narrow query blocks keep their logits (rows_pad floats per token, at most 1/4 of the K bytes) so that
     // the usage pass need not read K again
     y.logits = off;     off = align_up(off + (y.rows_pad_cap <= 16 && c->max_window > 0 ? U * T * (size_t)y.rows_pad_cap * 4 : 0), 256);
-    y.ctrl = off;       off = align_up(off + U * 2 * 4, 256);
     y.qctrl = off;      off = align_up(off + (size_t)(4 + c->n_layers * c->max_batch) * 4, 256);
-    y.finz = off;       off = align_up(off + U * 128 * 4, 256);
     y.total = off;
     return y;
 }
@@ -182,8 +180,12 @@ int ams_init_state(const ams_config *cfg, void *ema_state, void *workspace, size
     if (workspace_bytes < lay.total) return AMS_ERR_CAPACITY;
     cudaStream_t s = (cudaStream_t)stream;
     if (cudaMemsetAsync(ema_state, 0, ams_ema_state_bytes(cfg), s) != cudaSuccess) return AMS_ERR_CUDA;
-    if (cudaMemsetAsync(workspace, 0, 256, s) != cudaSuccess) return AMS_ERR_CUDA;
-    if (cudaMemsetAsync((unsigned char *)workspace + lay.ctrl, 0, lay.total - lay.ctrl, s) != cudaSuccess) return AMS_ERR_CUDA;
+    // status word, effective lengths and error flags; kept positions and segment counts start from zero so that
+    // nothing downstream ever indexes with an uninitialised value
+    if (cudaMemsetAsync(workspace, 0, lay.scores, s) != cudaSuccess) return AMS_ERR_CUDA;
+    if (cudaMemsetAsync((unsigned char *)workspace + lay.n_seg, 0, lay.raw_cuts - lay.n_seg, s) != cudaSuccess) return AMS_ERR_CUDA;
+    if (cudaMemsetAsync((unsigned char *)workspace + lay.keep_idx, 0, lay.part - lay.keep_idx, s) != cudaSuccess) return AMS_ERR_CUDA;
+    if (cudaMemsetAsync((unsigned char *)workspace + lay.qctrl, 0, lay.total - lay.qctrl, s) != cudaSuccess) return AMS_ERR_CUDA;
     ams_state *st = new (std::nothrow) ams_state;
     if (!st) return AMS_ERR_INTERNAL;
     st->cfg = *cfg;
@@ -236,7 +238,9 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
     p.fixed_seg = c.fixed_segments; p.uniform_q = c.uniform_quotas;
     p.lambda = c.ema_lambda; p.beta = c.ema_beta; p.eps = c.eps;
     p.k_pages = (__nv_bfloat16 *)k_pages; p.v_pages = (__nv_bfloat16 *)v_pages; p.num_pages = num_pages;
-    p.block_table = block_table; p.bt_stride = block_table_stride; p.seq_lens = seq_lens;
+    p.block_table = block_table; p.bt_stride = block_table_stride;
+    p.seq_lens = (const int *)(st->ws + y.eff_lens); p.seq_lens_out = seq_lens;
+    p.seq_bad = (int *)(st->ws + y.seq_bad);
     p.q = (const __nv_bfloat16 *)obs_queries; p.ema = (float *)ema_state; p.dst_pages = dst_pages;
     p.scores = (float *)(st->ws + y.scores);
     p.usage = p.scores;
@@ -248,6 +252,7 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
     p.cbuf = (u64 *)(st->ws + y.cbuf); p.flags = st->ws + y.flags;
     p.n_seg = (int *)(st->ws + y.n_seg); p.seg_bounds = (int *)(st->ws + y.seg_bounds);
     p.quotas = (int *)(st->ws + y.quotas); p.keep_idx = (int *)(st->ws + y.keep_idx);
+    p.raw_cuts = (int *)(st->ws + y.raw_cuts);
     p.mass_dbg = dbg ? dbg->mass : nullptr;
     p.part = (float *)(st->ws + y.part); p.fin = (float *)(st->ws + y.fin);
     p.slice_len = y.slice_len; p.n_slices = y.n_slices;
@@ -255,9 +260,6 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
     p.tc_tpc_min = tc_tiles_per_block_min(y.T_cap);
     p.tc_stages = p.rows_pad <= 256 ? 4 : 2; // even: each stage then belongs to one of the two MMA issuers
     p.status = (int *)(st->ws + y.status);
-    p.fcnt = (int *)(st->ws + y.ctrl);
-    p.fflag = p.fcnt + (size_t)c.n_layers * c.max_batch * c.n_kv_heads;
-    p.finz = (float *)(st->ws + y.finz);
     p.qctrl = (int *)(st->ws + y.qctrl);
     p.logits = (y.rows_pad_cap <= 16 && c.max_window > 0) ? (float *)(st->ws + y.logits) : nullptr;
 
@@ -267,9 +269,13 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
     ctx.ev = st->profiling ? st->ev : nullptr;
     ctx.max_ev = 32;
     ctx.begin();
-    if (scorer_id == AMS_SCORER_TOVA) {
+    // lengths and page ids are checked once, on the device, before anything forms an address from them
+    p.W = (scorer_id == AMS_SCORER_TOVA || split) ? window : 0;
+    rc = launch_prepare(p, seq_lens, (int *)(st->ws + y.eff_lens), ctx);
+    p.W = scorer_id == AMS_SCORER_TOVA ? window : 0;
+    if (rc == AMS_OK && scorer_id == AMS_SCORER_TOVA) {
         rc = launch_score_tova(p, ctx);
-    } else if (scorer_id == AMS_SCORER_KEYDIFF) {
+    } else if (rc == AMS_OK && scorer_id == AMS_SCORER_KEYDIFF) {
         if (split) {
             // the window attention goes through the score array into the usage array (smoothed on the way
             // if asked for); the key-only score then takes the score array
@@ -288,8 +294,12 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
         rc = launch_smooth_usage(p, p.usage, usage_buf, c.pool_kernel, ctx);
         p.usage = usage_buf;
     }
-    const bool queued = segment_moves_rows(p); // the work-queue form of the segmentation kernel starts the compaction
-    if (rc == AMS_OK) rc = segment_cluster_supported(p) ? launch_segment_select_cluster(p, ctx) : launch_segment_select(p, ctx);
+    bool queued = false;
+    if (rc == AMS_OK) {
+        if (segsel_supported(p)) rc = launch_segsel(p, ctx);
+        else if (segment_cluster_supported(p)) { queued = segment_moves_rows(p); rc = launch_segment_select_cluster(p, ctx); }
+        else rc = launch_segment_select(p, ctx);
+    }
     if (rc == AMS_OK && dbg) {
         // inspection copies are taken before the table is rewritten
         const size_t U = (size_t)p.L * p.B * p.H;
@@ -320,6 +330,12 @@ int ams_get_status(ams_state *st, void *stream, int32_t *detail)
     if (cudaStreamSynchronize(s) != cudaSuccess) return AMS_ERR_CUDA;
     if (detail) memcpy(detail, host, sizeof host);
     return host[0];
+}
+
+int ams_debug_expire_wait(ams_state *st, uint32_t polls, void *stream)
+{
+    if (!st || polls < 1 || polls > (1u << 20)) return AMS_ERR_INVALID_ARG;
+    return launch_expire_wait((int *)(st->ws + st->lay.status), polls, (cudaStream_t)stream);
 }
 
 int32_t ams_last_launch_count(const ams_state *st) { return st ? st->last_launches : 0; }
@@ -357,7 +373,7 @@ int ams_get_kernel_times(ams_state *st, float *ms)
 const char *ams_kernel_name(int32_t idx)
 {
     static const char *names[kKernCount] = {"score_phase1", "score_combine", "score_phase2", "segment_select",
-                                            "gather", "table_update", "usage_signal"};
+                                            "gather", "table_update", "usage_signal", "prepare", "segments_quotas", "select_compact"};
     return idx >= 0 && idx < kKernCount ? names[idx] : nullptr;
 }
 

@@ -29,7 +29,10 @@ struct DevParams {
     long long num_pages;
     int *block_table;
     int bt_stride;
-    int *seq_lens;
+    const int *seq_lens;              // effective lengths of this call ([B], workspace): the caller's length where the
+                                      // sequence is compressed, 0 where it is skipped (within the budget) or was
+                                      // reported (over capacity, window longer than the sequence, bad page id)
+    int *seq_lens_out;                // the caller's lengths, rewritten by the table update
     const __nv_bfloat16 *q;           // [L][B][H*G][W][128]
     float *ema;                       // [L][Bmax][H][T_cap]
     const int *dst_pages;             // [B][n_dst]
@@ -42,6 +45,7 @@ struct DevParams {
     int *seg_bounds;                  // [seg_cap + 1]
     int *quotas;                      // [seg_cap]
     int *keep_idx;                    // [Tk]
+    int *raw_cuts;                    // [S + 1]  cut after the token that reaches mass quantile k (T: none)
     float *mass_dbg;                  // [T_cap] or null
     // scorer scratch
     float *part;                      // per (unit, slice) partials
@@ -49,10 +53,9 @@ struct DevParams {
     int slice_len, n_slices, rows_pad;
     int tc_tpc_min, tc_stages;        // tensor-core scorer: least tiles per block, K stages in shared memory
     int tc_hpb;                       // tensor-core scorer: KV heads a block takes one after the other (set by its launcher)
-    int *fcnt, *fflag;                // fused scorer: per-unit counters of tiles in / of query rows merged ([2][units], contiguous)
-    float *finz;                      // fused scorer: 1 / Z_r per unit and query row, [units][rows_pad]
     int *qctrl;                       // work-queue counters of the one-block segmentation kernel, [4 + L * Bmax], zero between events
     float *logits;                    // narrow query blocks (rows_pad <= 16): scaled logits [units][T_cap][rows_pad], or null
+    int *seq_bad;                     // [B]: set when a unit of the sequence reported a device-side error (its rows stay)
     int *status;                      // [4]: code, unit, a, b
 };
 
@@ -202,7 +205,7 @@ inline cudaError_t launch_after(void (*kernel)(KArgs...), dim3 grid, dim3 block,
 
 // Host-side launchers (one per translation unit).
 int tova_rows_block(int rows); // query rows handled per pass of the TOVA kernel (8..128)
-enum KernelId { kKernScore1 = 0, kKernScoreCombine, kKernScore2, kKernSegmentSelect, kKernGather, kKernTable, kKernUsage, kKernCount };
+enum KernelId { kKernScore1 = 0, kKernScoreCombine, kKernScore2, kKernSegmentSelect, kKernGather, kKernTable, kKernUsage, kKernPrepare, kKernQuota, kKernSelect, kKernCount };
 
 // Stream, launch counter and optional per-kernel timing events of one ams_compress call.
 struct LaunchCtx {
@@ -228,16 +231,48 @@ int launch_score_tova(const DevParams &p, LaunchCtx &ctx);
 bool tova_tc_supported(const DevParams &p);
 size_t tova_tc_smem_bytes(const DevParams &p);
 int launch_score_tova_tc(const DevParams &p, LaunchCtx &ctx);
-bool tova_fused_supported(const DevParams &p);
-int launch_score_tova_fused(const DevParams &p, LaunchCtx &ctx);
 int launch_score_keydiff(const DevParams &p, LaunchCtx &ctx);
 int launch_segment_select(const DevParams &p, LaunchCtx &ctx);
+bool segsel_supported(const DevParams &p);   // the three-kernel form of Algorithm 1 steps 1-5
+int launch_segsel(const DevParams &p, LaunchCtx &ctx);
 bool segment_cluster_supported(const DevParams &p);
 bool segment_moves_rows(const DevParams &p); // the segmentation launch also starts the paged compaction
 int launch_segment_select_cluster(const DevParams &p, LaunchCtx &ctx);
 constexpr int kMoveRows = 512; // (token, head) rows of K and V per chunk of the paged compaction
 int launch_gather(const DevParams &p, LaunchCtx &ctx, bool queued); // queued: chunks below p.qctrl[1] are moved already
 int launch_smooth_usage(const DevParams &p, const float *src, float *dst, int k, LaunchCtx &ctx);
+// First kernel of an event: validates lengths and page ids, writes the effective lengths (lens_in: the caller's).
+int launch_prepare(const DevParams &p, const int *lens_in, int *eff_lens, LaunchCtx &ctx);
+int launch_expire_wait(int *status, uint32_t polls, cudaStream_t s); // test hook: a bounded wait that runs out
+
+// Launch state that differs per device (one process may drive several GPUs): SM count and, per kernel, the
+// dynamic shared-memory limit already granted.
+constexpr int kMaxDevices = 64;
+inline int current_device()
+{
+    int d = -1;
+    return (cudaGetDevice(&d) == cudaSuccess && d >= 0 && d < kMaxDevices) ? d : -1;
+}
+inline int sm_count()
+{
+    static int n_sm[kMaxDevices];
+    const int d = current_device();
+    if (d < 0) return 0;
+    if (!n_sm[d] && cudaDeviceGetAttribute(&n_sm[d], cudaDevAttrMultiProcessorCount, d) != cudaSuccess) n_sm[d] = 0;
+    return n_sm[d];
+}
+struct SmemGrant { size_t bytes[kMaxDevices]; };
+template <typename K>
+inline bool grant_dynamic_smem(K kernel, size_t smem, SmemGrant &g)
+{
+    const int d = current_device();
+    if (d < 0) return false;
+    if (smem > g.bytes[d]) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return false;
+        g.bytes[d] = smem;
+    }
+    return true;
+}
 int launch_retained_iou(const DevParams &p, const int *prev_kept, float *out, LaunchCtx &ctx); // before the lengths are rewritten
 
 } // namespace ams

@@ -26,7 +26,7 @@ __global__ void __launch_bounds__(kGatherThreads) k_gather(DevParams p, int queu
     }
     const int b = lb % p.B, l = lb / p.B;
     const int T = p.seq_lens[b];
-    if (T <= p.Tk || T > p.T_cap) return;
+    if (T <= p.Tk || T > p.T_cap || p.seq_bad[b]) return;
     const int n_rows = p.Tk * p.H;
     const int lane = threadIdx.x & 15, rsub = threadIdx.x >> 4;
     const int r0 = blockIdx.x * kRowsPerBlock + rsub;
@@ -66,14 +66,12 @@ __global__ void k_table_update(DevParams p)
     wait_for_previous_kernel(); // the gather kernel reads the table this kernel rewrites
     const int b = blockIdx.x;
     const int T = p.seq_lens[b];
-    if (T <= p.Tk || T > p.T_cap) return;
+    if (T <= p.Tk || T > p.T_cap || p.seq_bad[b]) return;
     int *row = p.block_table + (size_t)b * p.bt_stride;
     for (int i = threadIdx.x; i < p.bt_stride; i += blockDim.x)
         row[i] = i < p.n_dst ? p.dst_pages[(size_t)b * p.n_dst + i] : -1;
-    if (b == 0) // work-queue counters of the segmentation kernel back to zero for the next event
-        for (int i = threadIdx.x; i < 4 + p.L * p.B; i += blockDim.x) p.qctrl[i] = 0;
     __syncthreads();
-    if (threadIdx.x == 0) p.seq_lens[b] = p.Tk;
+    if (threadIdx.x == 0) p.seq_lens_out[b] = p.Tk;
 }
 
 } // namespace

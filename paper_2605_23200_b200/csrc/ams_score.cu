@@ -418,7 +418,6 @@ int tova_rows_block(int rows)
 
 int launch_score_tova(const DevParams &p, LaunchCtx &ctx)
 {
-    if (tova_fused_supported(p)) return launch_score_tova_fused(p, ctx);
     if (tova_tc_supported(p)) return launch_score_tova_tc(p, ctx);
     switch (tova_rows_block(p.rows) / 8) {
     case 1: launch_tova_ntb<1>(p, ctx); break;

@@ -485,19 +485,11 @@ int launch_score_tova_tc(const DevParams &p_in, LaunchCtx &ctx)
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return AMS_ERR_CUDA;
     }
-    static int n_sm = 0;
-    if (!n_sm) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return AMS_ERR_CUDA;
-    }
+    const int n_sm = sm_count();
+    if (n_sm <= 0) return AMS_ERR_CUDA;
     const size_t smem = tova_tc_smem_bytes(p);
-    static size_t configured = 0;
-    if (smem > configured) {
-        if (cudaFuncSetAttribute(k_tova_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
-            cudaFuncSetAttribute(k_tova_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-            return AMS_ERR_CUDA;
-        configured = smem;
-    }
+    static SmemGrant grant1, grant2;
+    if (!grant_dynamic_smem(k_tova_tc<1>, smem, grant1) || !grant_dynamic_smem(k_tova_tc<2>, smem, grant2)) return AMS_ERR_CUDA;
     const long long cap_tiles = (long long)p.L * p.B * ((p.T_cap + kTileTokens - 1) / kTileTokens); // per head
     long long want = (cap_tiles + p.tc_tpc_min - 1) / p.tc_tpc_min;
     // heads per block: the divisor of H that fills most SMs (the smallest one on a tie)

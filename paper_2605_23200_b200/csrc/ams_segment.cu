@@ -1,6 +1,8 @@
-// Mass, EMA credit, prefix scan, cuts, merge/split, quotas, segmented radix select,
-// must-keep, backfill and ordered index compaction: Algorithm 1 steps 1-5 of the
-// paper for one (layer, sequence, KV head) per thread block.
+// Mass, prefix scan, cuts, merge/split, quotas, segmented radix select, must-keep,
+// backfill and ordered index compaction: Algorithm 1 steps 1-5 of the paper for one
+// score row per thread block, with every per-token array in global scratch.  This
+// one-kernel form serves the allocation-free entry point at the end of the file (its
+// scratch is a fixed array); ams_compress uses the three kernels of ams_segsel.cu.
 //
 // Every decision is integer arithmetic on fixed-point images of the mass (kFixBits
 // fractional bits) and every floating-point step is a single round-to-nearest
@@ -328,12 +330,8 @@ int launch_segment_select(const DevParams &p, LaunchCtx &ctx)
     const int nthreads = 1024;
     const size_t dyn = (size_t)p.seg_cap * 8 + (size_t)(4 * p.seg_cap + 1) * 4 + (size_t)3 * (p.S + 1) * 4 +
                        (size_t)(nthreads / 32) * (256 + 4) * 4 + 64;
-    static size_t configured = 0;
-    if (dyn > configured) {
-        if (cudaFuncSetAttribute(k_segment_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
-            return AMS_ERR_CUDA;
-        configured = dyn;
-    }
+    static SmemGrant grant;
+    if (!grant_dynamic_smem(k_segment_select, dyn, grant)) return AMS_ERR_CUDA;
     k_segment_select<<<units, nthreads, dyn, ctx.s>>>(p);
     ctx.mark(kKernSegmentSelect);
     return cudaGetLastError() == cudaSuccess ? AMS_OK : AMS_ERR_CUDA;
@@ -349,7 +347,7 @@ int launch_segment_select(const DevParams &p, LaunchCtx &ctx)
 // a serving process whose memory pool is owned and fully reserved by the host framework, and
 // callers on a hot path that must not take the allocator's locks.  For them the scratch the
 // selection kernel needs lives in the fixed array below instead of a caller-supplied
-// workspace.  Every GPU that loads the library holds the array (kStaticBytes, about 2.6 MB)
+// workspace.  Every GPU that loads the library holds the array (kStaticBytes, about 2.4 MB)
 // until the process exits.
 namespace ams {
 namespace {
@@ -374,9 +372,8 @@ constexpr size_t kStaticBytes = StaticLayout::total;
 // In host code this name is only a handle for cudaGetSymbolAddress, never a device address.
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
 
-__global__ void k_static_prepare(int *status, int *lens, int n_units, int seq_len)
+__global__ void k_static_prepare(int *lens, int n_units, int seq_len)
 {
-    if (threadIdx.x < 4) status[threadIdx.x] = 0;
     if (threadIdx.x < n_units) lens[threadIdx.x] = seq_len;
 }
 
@@ -443,7 +440,27 @@ extern "C" int ams_select_static(const ams_config *cfg, const float *scores, int
     p.keep_idx = keep_idx;
     p.status = (int *)(base + StaticLayout::status);
 
-    k_static_prepare<<<1, 32, 0, s>>>(p.status, p.seq_lens, n_units, seq_len);
+    k_static_prepare<<<1, 32, 0, s>>>((int *)(base + StaticLayout::lens), n_units, seq_len);
     k_segment_select<<<n_units, nthreads, dyn, s>>>(p);
     return cudaGetLastError() == cudaSuccess ? AMS_OK : AMS_ERR_CUDA;
+}
+
+// Device-side conditions of the calls above (a segment table that overflowed, a count that did not add up)
+// land in a status word inside the same fixed array; this reads and clears it, like ams_get_status does
+// for a handle.  Copies 16 bytes, allocates nothing, synchronises `stream`.
+extern "C" int ams_select_static_status(int32_t *detail, void *stream)
+{
+    using namespace ams;
+    int32_t host[4] = {0, 0, 0, 0};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kStaticMaxDevices) return AMS_ERR_CUDA;
+    const PerDevice &pd = g_static_dev[dev];
+    if (pd.ready) {
+        cudaStream_t s = (cudaStream_t)stream;
+        if (cudaMemcpyAsync(host, pd.base + StaticLayout::status, sizeof host, cudaMemcpyDeviceToHost, s) != cudaSuccess) return AMS_ERR_CUDA;
+        if (cudaMemsetAsync(pd.base + StaticLayout::status, 0, sizeof host, s) != cudaSuccess) return AMS_ERR_CUDA;
+        if (cudaStreamSynchronize(s) != cudaSuccess) return AMS_ERR_CUDA;
+    }
+    if (detail) memcpy(detail, host, sizeof host);
+    return host[0];
 }

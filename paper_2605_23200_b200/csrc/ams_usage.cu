@@ -55,7 +55,72 @@ __global__ void __launch_bounds__(128) k_retained_iou(DevParams p, const int *pr
     out[uid] = either > 0 ? __fdiv_rn((float)both, (float)either) : 0.0f;
 }
 
+// First kernel of an event, one block per sequence: the effective length the other kernels work with.
+// A sequence within the budget has nothing to evict (effective length 0: every kernel skips it).  A
+// sequence over the configured capacity, shorter than the observation window, or whose block-table
+// row or replacement pages name a page outside the pool is reported through the status word and
+// skipped as well, so that no kernel ever forms an address from a bad page id.
+__global__ void __launch_bounds__(256) k_prepare(DevParams p, const int *lens_in, int *eff_lens)
+{
+    const int b = blockIdx.x;
+    const int T = lens_in[b];
+    int eff = 0;
+    if (T > p.Tk) {
+        if (T > p.T_cap) {
+            if (threadIdx.x == 0) set_status(p.status, AMS_ERR_CAPACITY, b, T, p.T_cap);
+        } else if (p.W > T) {
+            if (threadIdx.x == 0) set_status(p.status, AMS_ERR_INVALID_ARG, b, p.W, T);
+        } else {
+            const int n_src = (T + kPage - 1) / kPage;
+            int bad = n_src > p.bt_stride ? 1 : 0;
+            const int *row = p.block_table + (size_t)b * p.bt_stride;
+            for (int i = threadIdx.x; i < n_src && !bad; i += blockDim.x) {
+                const int pg = row[i];
+                if (pg < 0 || (long long)pg >= p.num_pages) { bad = 1; set_status(p.status, AMS_ERR_INVALID_ARG, b, i, pg); }
+            }
+            for (int i = threadIdx.x; i < p.n_dst; i += blockDim.x) {
+                const int pg = p.dst_pages[(size_t)b * p.n_dst + i];
+                if (pg < 0 || (long long)pg >= p.num_pages) { bad = 1; set_status(p.status, AMS_ERR_INVALID_ARG, b, -1 - i, pg); }
+            }
+            if (!__syncthreads_or(bad)) eff = T;
+        }
+    }
+    if (threadIdx.x == 0) { eff_lens[b] = eff; p.seq_bad[b] = 0; }
+}
+
+// Test hook: one thread waits on an mbarrier that nobody will ever arrive at, gives up after `polls`
+// polls and reports AMS_ERR_TIMEOUT through the status word, exactly as the bounded waits of the
+// tensor-core scorer do.  Nothing else is touched; the context stays usable.
+__global__ void k_expire_wait(int *status, uint32_t polls)
+{
+    __shared__ unsigned long long bar;
+    const uint32_t addr = (uint32_t)__cvta_generic_to_shared(&bar);
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(addr), "r"(1) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    bool done = false;
+    for (uint32_t i = 0; i < polls && !done; ++i) {
+        uint32_t ok;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(addr), "r"(0) : "memory");
+        done = ok != 0;
+    }
+    if (!done) set_status(status, AMS_ERR_TIMEOUT, -1, (int)polls, 0);
+}
+
 } // namespace
+
+int launch_prepare(const DevParams &p, const int *lens_in, int *eff_lens, LaunchCtx &ctx)
+{
+    k_prepare<<<p.B, 256, 0, ctx.s>>>(p, lens_in, eff_lens);
+    ctx.mark(kKernPrepare);
+    return cudaGetLastError() == cudaSuccess ? AMS_OK : AMS_ERR_CUDA;
+}
+
+int launch_expire_wait(int *status, uint32_t polls, cudaStream_t s)
+{
+    k_expire_wait<<<1, 1, 0, s>>>(status, polls);
+    return cudaGetLastError() == cudaSuccess ? AMS_OK : AMS_ERR_CUDA;
+}
 
 int launch_retained_iou(const DevParams &p, const int *prev_kept, float *out, LaunchCtx &ctx)
 {

@@ -30,7 +30,7 @@ def test_benchmark_workload_sampled_units_and_properties():
     v_before = cache.v_pages.clone()
     dst = inputs.alloc_dst_pages(cache)
     dbg = gpu_event(comp, cache, dst)
-    assert comp.last_launch_count == 5          # the launch sequence bench.py times
+    assert comp.last_launch_count == 8          # validation, two scorer passes, three selection kernels, gather, table
     got = dbg.scores.cpu().numpy()
     mass = dbg.mass.cpu().numpy()
     T, Tk, G = wl.seq_len_max, wl.budget, wl.group

@@ -56,8 +56,7 @@ def test_smoothed_external_usage_bit_exact(k, kw):
     credit0 = comp.ema_state.cpu().numpy()
     dst = inputs.alloc_dst_pages(cache)
     dbg = gpu_event(comp, cache, dst, inputs.SCORER_EXTERNAL, torch.from_numpy(ext).to(DEV))
-    n_classes = 1 if wl.max_seq_len <= 16384 else 2          # one segment/select launch per cluster size
-    assert comp.last_launch_count == 3 + n_classes           # smoothing, segment/select, gather, table update
+    assert comp.last_launch_count == 7           # validation, smoothing, three selection kernels, gather, table update
     _usage_rows_equal(dbg, snap, wl, lambda l, b, h, T: oracle.smooth_usage(ext[l, b, h, :T], k))
     compare_event(snap, cache, comp, dbg, dst, credit0, ext, pool_kernel=k)
 

@@ -1,11 +1,12 @@
-"""The allocation-free selection entry point (`ams_select_static`) against the regular one.
+"""The allocation-free selection entry point (`ams_select_static`) against the regular one and the oracle.
 
 Some users of the library cannot allocate device memory where they call it — a stream capture
 is in progress, or the process's device memory pool belongs to the framework that hosts them —
 so this entry point works out of a fixed scratch array inside the library.  The check: on the
 same scores it must keep exactly the positions that `ams_compress` keeps (external-score mode,
-credit off), on two calls in a row, the second one on different scores so that anything left in
-the shared scratch by the first call would show.  Collected last on purpose."""
+credit off) and that the CPU oracle keeps, on calls in a row: the second one on different scores,
+the third one with fewer and shorter rows, so that anything left in the shared scratch by an
+earlier, larger call would show.  Collected last on purpose."""
 import ctypes
 import gc
 
@@ -13,6 +14,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2605_23200_b200 import binding, inputs
 
 pytestmark = pytest.mark.gpu
@@ -56,6 +58,20 @@ def test_static_scratch_selection_matches_regular_entry_point_twice():
         assert torch.cuda.memory_allocated() <= allocated
         assert torch.cuda.mem_get_info()[0] >= free_before - (64 << 20)
         assert torch.equal(got, want), f"call {call}"
+        prm = oracle.Params(wl.n_segments, wl.l_min, wl.l_max, wl.q_min, wl.n_sink, wl.n_last, wl.ema_lambda, 1.0, wl.eps)
+        for r in range(8):
+            assert (got[r].cpu().numpy() == oracle.select_unit(x[0, 0, r, :T], None, None, Tk, prm).keep_idx).all(), (call, r)
+        assert binding.select_static_status() == (binding.AMS_OK, [0, 0, 0, 0])
+    # third call: fewer rows, a shorter sequence and another stride than the calls before it
+    T3, Tk3, stride3 = 1203, 200, 1216
+    x3 = np.exp(rng.standard_normal((3, stride3))).astype(np.float32)
+    got3 = torch.full((3, Tk3), -1, dtype=torch.int32, device=DEV)
+    binding.select_static(cfg, torch.from_numpy(x3).to(DEV), T3, Tk3, 7, got3)
+    torch.cuda.synchronize()
+    prm3 = oracle.Params(7, wl.l_min, wl.l_max, wl.q_min, wl.n_sink, wl.n_last, wl.ema_lambda, 1.0, wl.eps)
+    for r in range(3):
+        assert (got3[r].cpu().numpy() == oracle.select_unit(x3[r, :T3], None, None, Tk3, prm3).keep_idx).all(), r
+    assert binding.select_static_status()[0] == binding.AMS_OK
 
 
 def test_static_scratch_limits_are_rejected():
