@@ -1,28 +1,36 @@
 #!/usr/bin/env python
 """Benchmark of the AMS compression step (score + segment + select + compact).
 
-One "step" is one `ams_compress` call over the whole layer stack of the workload.
-At N = 1 the workload is benchmark configuration 1 (Llama-3.1-8B-shaped stack:
-32 layers, 32 q / 8 KV heads, d = 128, one sequence of 16384 cached bf16 tokens in
-16-token pages, compressed to 2048; observation window 32, TOVA-style scorer).
-With N > 1 every rank runs its own replica of that workload (the units of the path
-are independent: no collective on the data path; weak scaling).
+One "step" is one `ams_compress` call over the whole layer stack of a workload.
 
-Prints ONE JSON line (rank 0).  `value` = whole-job steps/s with the cache resident in
-HBM, timed with CUDA events on the launching stream.  `e2e` = the same through the
-C ABI with the step's inputs (observation queries, block table, lengths,
-replacement pages) copied from pinned host memory and its results (block table,
-lengths) read back and checked inside the timed region; the upload of the next
-step's inputs and the read-back of the previous step's results overlap the current
-step's kernels (three buffer sets, at most two steps in flight), as a serving loop
-would do; the paged K/V pool is the persistent device
-state the step operates on and is not copied.
+Headline (`value`, `ms_per_step`, `roofline`, `e2e`, `cpu_baseline`): the largest of the five
+benchmark configurations that fits one GPU, configuration 4 (Llama-3.1-70B-shaped stack: 80 layers,
+64 q / 8 KV heads, one sequence of 131072 cached bf16 tokens in 16-token pages compressed to 8192,
+observation window 64, 32 mass quantiles), first event.  `per_config` then carries all five
+configurations, each timed in the same process on freshly generated inputs: first event, and for
+the two multi-event configurations (2: 20 events with 128 appended tokens; 4: 8 events with 512)
+the steady-state events 2..N run as real successive events with the EMA state carried.
+Configuration 3 (309 GB of K/V) does not fit: four of its 36 layers are resident and one launch
+covers those four; its figures are per such launch.
+
+With N > 1 every rank runs its own replica of the workload (the units of the path are independent:
+no collective on the data path; weak scaling).  `--gpus N` without a launcher spawns the N ranks
+itself; under torchrun it must agree with WORLD_SIZE.
+
+Prints ONE JSON line (rank 0).  `value` = whole-job steps/s with the cache resident in HBM, timed
+with CUDA events on the launching stream.  `e2e` = the same through the C ABI with the step's
+inputs (observation queries, block table, lengths, replacement pages) copied from pinned host
+memory and its results (block table, lengths) read back and checked inside the timed region; the
+paged K/V pool is the persistent device state the step operates on and is not copied.
 """
 from __future__ import annotations
 
 import argparse
+import gc
 import json
 import os
+import socket
+import subprocess
 import sys
 import threading
 import time
@@ -36,6 +44,10 @@ import torch
 
 METRIC = "ams_compress_steps_per_s"
 UNIT = "steps/s"
+HEADLINE_CFG = 4
+L2_BYTES = 126 << 20
+MUFU_PER_CLK_PER_SM = 16          # special-function results per clock and SM (exp2)
+N_SM = 148
 
 
 def _peaks():
@@ -43,19 +55,26 @@ def _peaks():
     if os.path.exists(path):
         with open(path) as f:
             d = json.load(f)
-        return float(d["hbm_gbs"]), "measured"
-    return 6650.0, "fallback"
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d.get("bf16_tflops", 1590.0)),
+                "sm_max_mhz": float(d.get("sm_max_mhz", 1965.0)), "kind": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "sm_max_mhz": 1965.0, "kind": "fallback"}
 
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the scorer passes on the
-# default workload, from the ncu capture summarised in profiles/kernels_cfg1_8layers_ncu_full.md: taken on
-# the 8-layer reduction of the workload and scaled x4 to the 32-layer launch (units are independent and each
-# is read once per pass).  Valid for that workload and the kernels as profiled; anything else reports null.
-NCU_TRAFFIC_BYTES = {
-    "cfg1_llama8b_L32_T16384_k2048_w32": {"score_phase1": 4 * (271_291_904 + 9_388_288),
-                                          "score_phase2": 4 * (271_763_712 + 7_136_256),
-                                          "gather": None},
-}
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch from ncu captures summarised under
+# profiles/ (workload -> kernel slot -> bytes per launch).  A kernel or workload without a capture of the
+# current code reports null.
+NCU_TRAFFIC_BYTES: dict = {}
+
+
+def config_dict(wl) -> dict:
+    """What defines the workload of a line (the same for both arms)."""
+    why = ("largest of the five configurations that fits one GPU (configuration 3 needs 309 GB)" if wl.cfg_id == HEADLINE_CFG
+           else "chosen with --config")
+    return {"workload": wl.name, "layers": wl.n_layers, "layers_resident": wl.layers_resident, "q_heads": wl.n_q_heads,
+            "kv_heads": wl.n_kv_heads, "batch_per_gpu": wl.batch, "cache_tokens": wl.seq_len_max, "budget": wl.budget,
+            "window": wl.window, "n_segments": wl.n_segments, "scorer": "tova" if wl.scorer_id == 0 else "keydiff",
+            "event": "first event (cache at full length); steady-state events are under per_config",
+            "why_this_workload": why}
 
 
 def algorithmic_bytes(wl, lens) -> tuple[int, int]:
@@ -130,105 +149,224 @@ def barrier():
         dist.barrier()
 
 
-def run_ours(args, rank, world, local_rank):
-    from paper_2605_23200_b200 import binding, build, inputs
-    import torch.distributed as dist
+class Bench:
+    """One workload instance on one device: cache, compressor and the pieces the timing loops need."""
 
-    if rank == 0:
-        build.build()
-    dev = torch.device(f"cuda:{local_rank}")
-    torch.cuda.set_device(dev)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-        barrier()
-    binding.lib()
-    wl = inputs.CONFIGS[args.config]
-    if args.layers:
-        wl = wl.scaled(n_layers=args.layers, resident_layers=0, name=wl.name + f"_REDUCED_to_{args.layers}_layers")
-    cache = inputs.make_cache(wl, dev)
-    comp = binding.AmsCompressor(binding.config_for(wl), dev)
-    stream = torch.cuda.current_stream(dev)
-    dst_np = inputs.alloc_dst_pages(cache)
-    dst = torch.from_numpy(dst_np).to(dev)
-    table0, lens0 = cache.block_table.clone(), cache.seq_lens.clone()
-    q = cache.obs_queries if wl.scorer_id == inputs.SCORER_TOVA else None
+    def __init__(self, cfg_id, dev, layers=0):
+        from paper_2605_23200_b200 import binding, inputs
+        self.inputs, self.binding = inputs, binding
+        wl = inputs.CONFIGS[cfg_id]
+        if layers:
+            wl = wl.scaled(n_layers=layers, resident_layers=0, name=wl.name + f"_REDUCED_to_{layers}_layers")
+        self.wl, self.dev = wl, dev
+        self.cache = inputs.make_cache(wl, dev)
+        self.comp = binding.AmsCompressor(binding.config_for(wl), dev)
+        self.stream = torch.cuda.current_stream(dev)
+        self.dst_np = inputs.alloc_dst_pages(self.cache)
+        self.dst = torch.from_numpy(self.dst_np).to(dev)
+        self.table0, self.lens0 = self.cache.block_table.clone(), self.cache.seq_lens.clone()
+        self.q = self.cache.obs_queries if wl.scorer_id == inputs.SCORER_TOVA else None
+        k_read, moved = algorithmic_bytes(wl, self.lens0.cpu().numpy())
+        self.k_read, self.moved = k_read, moved
+        # inputs smaller than twice the L2 are flushed out of it between timed steps
+        self.flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev) if k_read < 2 * L2_BYTES else None
 
-    def restore():
-        cache.block_table.copy_(table0)
-        cache.seq_lens.copy_(lens0)
-        comp.ema_state.zero_()
+    def restore(self):
+        self.cache.block_table.copy_(self.table0)
+        self.cache.seq_lens.copy_(self.lens0)
+        self.comp.ema_state.zero_()
+        if self.flush is not None:
+            self.flush.fill_(1)
 
-    def step():
-        comp.compress(cache.k_pages, cache.v_pages, cache.block_table, cache.seq_lens, q, wl.budget, wl.n_segments,
-                      wl.scorer_id, dst)
+    def step(self):
+        wl, c = self.wl, self.cache
+        self.comp.compress(c.k_pages, c.v_pages, c.block_table, c.seq_lens, self.q, wl.budget, wl.n_segments,
+                           wl.scorer_id, self.dst)
 
-    def timed(n, body):
+    def timed(self, n, body):
         evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
         for a, b in evs:
-            restore()
-            a.record(stream)
+            self.restore()
+            a.record(self.stream)
             body()
-            b.record(stream)
-        torch.cuda.synchronize(dev)
+            b.record(self.stream)
+        torch.cuda.synchronize(self.dev)
         return [a.elapsed_time(b) for a, b in evs]
 
-    for _ in range(max(args.warmup, 3)):
-        restore()
-        step()
-    comp.status()
-    torch.cuda.synchronize(dev)
-    direct_step = step
-    if args.graph:
-        # the whole step as one CUDA graph launch (pays off where the step is launch-bound)
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph):
-            direct_step()
-        restore()
-        step = graph.replay
-        stream = torch.cuda.current_stream(dev)
-        for _ in range(3):
-            restore()
-            step()
+    def warm(self, n):
+        for _ in range(max(n, 3)):
+            self.restore()
+            self.step()
+        self.comp.status()
+        torch.cuda.synchronize(self.dev)
+
+    def kernel_times(self, n):
+        self.comp.set_profiling(True)
+        acc = {}
+        for _ in range(n):
+            self.restore()
+            self.step()
+            for k, v in self.comp.kernel_times_ms().items():
+                acc[k] = acc.get(k, 0.0) + v
+        self.comp.set_profiling(False)
+        return {k: v / n for k, v in acc.items() if v > 0.0}      # a slot no kernel of this path used stays out
+
+    def close(self):
+        self.comp.close()
+        for name in ("cache", "comp", "dst", "table0", "lens0", "q", "flush"):
+            setattr(self, name, None)
+        gc.collect()
+        torch.cuda.empty_cache()
+
+
+SCORE_SLOTS = ("score_phase1", "score_combine", "score_phase2")
+SELECT_SLOTS = ("segment_select", "segments_quotas", "select_compact")
+
+
+def roofline_of(wl, kern_ms, k_read, moved, lens, peaks, traffic=None):
+    """Roofline object of the dominant kernel that has an algorithmic byte (or operation) count: the scorer
+    passes (K bytes; exponentials and tensor flops when the query block is wide) and the gather (kept rows).
+    The selection kernels read no K/V byte; if one of them is the longest kernel the note says so."""
+    if not kern_ms:
+        return None
+    overall = max(kern_ms, key=kern_ms.get)
+    cands = {k: v for k, v in kern_ms.items() if k in ("score_phase1", "score_phase2", "gather")}
+    dom = max(cands, key=cands.get)
+    ms = cands[dom]
+    rows = wl.group * max(wl.window, 1)
+    note = []
+    if overall != dom:
+        note.append(f"longest kernel of the step is {overall} ({kern_ms[overall]:.4f} ms), which moves no K/V byte; the roofline is "
+                    f"quoted for the longest kernel that does")
+    if dom == "gather":
+        bytes_launch, bound = moved, "hbm"
+    else:
+        bytes_launch = k_read
+        # wide query blocks: two passes with one exponential and one multiply-add per (row, token, d) each; the
+        # special-function unit is the ceiling that binds first from about 75 rows, the tensor pipe next
+        bound = "alu" if (wl.scorer_id == 0 and rows >= 256) else "hbm"
+    out = {"kernel": dom, "bound": bound, "peak_kind": peaks["kind"], "algorithmic_bytes_per_launch": bytes_launch,
+           "traffic": (traffic or {}).get(dom)}
+    hbm_achieved = bytes_launch / (ms * 1e-3) / 1e9
+    if bound == "hbm":
+        out.update(achieved=hbm_achieved, peak=peaks["hbm_gbs"], unit="GB/s", frac=hbm_achieved / peaks["hbm_gbs"])
+        note.append("achieved = algorithmic bytes of the launch / mean CUDA-event duration of that kernel; frac is of the measured copy bandwidth")
+    else:
+        token_heads = wl.layers_resident * wl.n_kv_heads * sum(int(t) for t in lens if int(t) > wl.budget)
+        exps = token_heads * rows
+        flops = exps * 2 * 128
+        mufu_peak = N_SM * MUFU_PER_CLK_PER_SM * peaks["sm_max_mhz"] * 1e6 / 1e9        # G results / s
+        achieved = exps / (ms * 1e-3) / 1e9
+        out.update(achieved=achieved, peak=mufu_peak, unit="Gexp/s", frac=achieved / mufu_peak,
+                   operations_per_launch=exps,
+                   also={"hbm_gbs": hbm_achieved, "hbm_frac": hbm_achieved / peaks["hbm_gbs"],
+                         "tensor_tflops": flops / (ms * 1e-3) / 1e12,
+                         "tensor_frac": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"]})
+        note.append("512 query rows per KV head: the pass takes one exp2 per (row, token) on the special-function unit "
+                    "(16 results per clock and SM x 148 SMs x the maximum SM clock = peak) and is bound by it before HBM; "
+                    "hbm and tensor fractions of the same launch are under 'also'")
+    out["note"] = "; ".join(note)
+    return out
+
+
+def steady_state(b: Bench):
+    """Events 2..N of a multi-event configuration, run as real successive events: the first event compresses
+    the long cache, then `append_per_step` tokens are appended and the cache is compressed again, the EMA
+    credit carried in the compressor's state.  Returns per-event times and the kernel split of the last."""
+    wl, cache, comp, inputs = b.wl, b.cache, b.comp, b.inputs
+    b.restore()
+    dst_np = b.dst_np
+    times = []
+    kern = {}
+    for ev in range(wl.steps):
+        if ev > 0:
+            inputs.append_tokens(cache, wl.append_per_step)
+            dst_np = inputs.alloc_dst_pages(cache)
+        dst = torch.from_numpy(dst_np).to(b.dev)
+        q = cache.obs_queries if wl.scorer_id == inputs.SCORER_TOVA else None
+        last = ev == wl.steps - 1
+        if last:
+            comp.set_profiling(True)
+        if b.flush is not None:
+            b.flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(b.stream)
+        comp.compress(cache.k_pages, cache.v_pages, cache.block_table, cache.seq_lens, q, wl.budget, wl.n_segments,
+                      wl.scorer_id, dst)
+        e1.record(b.stream)
+        torch.cuda.synchronize(b.dev)
+        times.append(e0.elapsed_time(e1))
+        if last:
+            kern = {k: v for k, v in comp.kernel_times_ms().items() if v > 0.0}
+            comp.set_profiling(False)
         comp.status()
-        torch.cuda.synchronize(dev)
-    barrier()
-    sampler = ClockSampler(local_rank)
-    sampler.start()
-    per_step = timed(args.steps, step)
-    barrier()
-    clocks = sampler.stop()
-    comp.status()
-    total_ms = max_over_ranks(float(sum(per_step)), dev)
-    launches = comp.last_launch_count * args.steps
+        assert bool((cache.seq_lens == wl.budget).all())
+        inputs.after_compress(cache, dst_np)
+    T = wl.budget + wl.append_per_step
+    units = wl.layers_resident * wl.batch * wl.n_kv_heads
+    bytes_ss = units * (T * 256 + wl.budget * 1024)
+    ss = times[1:]
+    ms = float(np.mean(ss))
+    return {"events": wl.steps, "appended_per_event": wl.append_per_step, "cache_tokens": T,
+            "first_event_ms": times[0], "steady_state_ms": ms, "steady_state_ms_min": float(np.min(ss)),
+            "algorithmic_bytes_per_step": bytes_ss, "effective_hbm_gbs": bytes_ss / (ms * 1e-3) / 1e9,
+            "effective_hbm_frac_of_8tbs": bytes_ss / (ms * 1e-3) / 8e12, "kernels_ms_last_event": kern}
 
-    # per-kernel durations (CUDA events recorded by the library after each launch, same stream)
-    comp.set_profiling(True)
-    n_prof = min(args.steps, 50)
-    acc = {}
-    for _ in range(n_prof):
-        restore()
-        direct_step()
-        for k, v in comp.kernel_times_ms().items():
-            acc[k] = acc.get(k, 0.0) + v
-    comp.set_profiling(False)
-    kern_ms = {k: v / n_prof for k, v in acc.items() if v > 0.0}      # a slot no kernel of this path used stays out
 
-    # end to end: per-step inputs from pinned host memory, results read back
+def measure_config(cfg_id, dev, steps, warmup, peaks, layers=0, with_steady=True):
+    """First-event timing (and steady state where the configuration has one) of one configuration."""
+    b = Bench(cfg_id, dev, layers)
+    wl = b.wl
+    b.warm(warmup)
+    per_step = b.timed(steps, b.step)
+    b.comp.status()
+    kern_ms = b.kernel_times(min(steps, 10))
+    ms = float(np.mean(per_step))
+    lens = b.lens0.cpu().numpy()
+    total = b.k_read + b.moved
+    entry = {
+        "workload": wl.name, "layers_resident": wl.layers_resident, "layers_total": wl.n_layers, "batch": wl.batch,
+        "kv_heads": wl.n_kv_heads, "query_rows_per_kv_head": wl.group * max(wl.window, 1),
+        "cache_tokens": [int(lens.min()), int(lens.max())], "budget": wl.budget, "n_segments": wl.n_segments,
+        "scorer": "tova" if wl.scorer_id == 0 else "keydiff", "steps": steps,
+        "ms_per_step": ms, "ms_per_step_min": float(np.min(per_step)), "steps_per_s": 1e3 / ms,
+        "algorithmic_bytes_per_step": total, "effective_hbm_gbs": total / (ms * 1e-3) / 1e9,
+        "effective_hbm_frac_of_8tbs": total / (ms * 1e-3) / 8e12,
+        "effective_hbm_frac_of_measured": total / (ms * 1e-3) / (peaks["hbm_gbs"] * 1e9),
+        "l2": "L2 flushed between timed steps (256 MB written)" if b.flush is not None else "inputs larger than L2",
+        "launches_per_step": b.comp.last_launch_count, "kernels_ms": kern_ms,
+        "roofline": roofline_of(wl, kern_ms, b.k_read, b.moved, lens, peaks, NCU_TRAFFIC_BYTES.get(wl.name)),
+    }
+    if wl.layers_resident != wl.n_layers:
+        entry["note"] = (f"{wl.layers_resident} of {wl.n_layers} layers resident (the whole stack's K/V does not fit one GPU): "
+                         f"all figures are per launch over the resident layers; the full stack is {wl.n_layers // wl.layers_resident} such launches")
+    if with_steady and wl.steps > 1:
+        entry["steady_state"] = steady_state(b)
+    return b, entry, per_step
+
+
+def e2e_loop(b: Bench, n_e2e):
+    """The step through the C ABI with its inputs uploaded from pinned host memory and its results read back
+    and checked every step; the upload of step i + 1 and the read-back of step i - 1 overlap the kernels of
+    step i (three buffer sets, three streams, at most two steps in flight)."""
+    wl, cache, comp, dev, stream = b.wl, b.cache, b.comp, b.dev, b.stream
+    q, dst = b.q, b.dst
+    b.restore()
     host_q = q.cpu().pin_memory() if q is not None else None
-    host_table, host_lens, host_dst = table0.cpu().pin_memory(), lens0.cpu().pin_memory(), dst.cpu().pin_memory()
+    host_table, host_lens, host_dst = b.table0.cpu().pin_memory(), b.lens0.cpu().pin_memory(), dst.cpu().pin_memory()
     out_table, out_lens = torch.empty_like(host_table).pin_memory(), torch.empty_like(host_lens).pin_memory()
     h2d = sum(t.numel() * t.element_size() for t in (host_q, host_table, host_lens, host_dst) if t is not None)
     d2h = out_table.numel() * 4 + out_lens.numel() * 4 + 16
-
-    # Two sets of device input buffers: while step i computes, the inputs of step i + 1 are uploaded on a second
-    # stream (what a serving loop does); every step still uploads all its inputs from pinned host memory, and
-    # its results (block table, lengths, device status) are read back and waited for before the next launch.
-    NB = 3  # buffer sets: one being uploaded, one computing, one being read back
+    NB = 3
     sets = [(q, cache.block_table, cache.seq_lens, dst)] + [
         (None if q is None else torch.empty_like(q), torch.empty_like(cache.block_table), torch.empty_like(cache.seq_lens),
          torch.empty_like(dst)) for _ in range(NB - 1)]
-    copy_stream = torch.cuda.Stream(dev)
+    copy_stream, read_stream = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
     uploaded = [torch.cuda.Event() for _ in range(NB)]
+    computed = [torch.cuda.Event() for _ in range(NB)]
+    read_back = [torch.cuda.Event() for _ in range(NB)]
+    outs = [(out_table, out_lens)] + [(torch.empty_like(out_table).pin_memory(), torch.empty_like(out_lens).pin_memory())
+                                      for _ in range(NB - 1)]
 
     def upload(i):
         qi, ti, li, di = sets[i % NB]
@@ -239,12 +377,6 @@ def run_ours(args, rank, world, local_rank):
             li.copy_(host_lens, non_blocking=True)
             di.copy_(host_dst, non_blocking=True)
             uploaded[i % NB].record(copy_stream)
-
-    read_stream = torch.cuda.Stream(dev)
-    computed = [torch.cuda.Event() for _ in range(NB)]
-    read_back = [torch.cuda.Event() for _ in range(NB)]
-    outs = [(out_table, out_lens)] + [(torch.empty_like(out_table).pin_memory(), torch.empty_like(out_lens).pin_memory())
-                                      for _ in range(NB - 1)]
 
     def check(i):                           # results of step i: wait for their read-back and look at them
         read_back[i % NB].synchronize()
@@ -265,62 +397,126 @@ def run_ours(args, rank, world, local_rank):
             outs[i % NB][1].copy_(li, non_blocking=True)
             read_back[i % NB].record(read_stream)
 
-    n_e2e = min(args.steps, 50)
-    e2e_ms = None
-    if not args.no_e2e:
-        torch.cuda.synchronize(dev)
-        upload(0)
-        for i in range(3):
-            e2e_step(i)
-        check(1)
-        check(2)
-        comp.status()
-        barrier()
-        t0 = time.perf_counter()
-        for i in range(3, 3 + n_e2e):
-            e2e_step(i)
-        check(1 + n_e2e)
-        check(2 + n_e2e)
-        comp.status()  # device status word of the whole run; synchronises the stream
-        torch.cuda.synchronize(dev)
-        e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3, dev)
+    torch.cuda.synchronize(dev)
+    upload(0)
+    for i in range(3):
+        e2e_step(i)
+    check(1)
+    check(2)
+    comp.status()
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(3, 3 + n_e2e):
+        e2e_step(i)
+    check(1 + n_e2e)
+    check(2 + n_e2e)
+    comp.status()  # device status word of the whole run; synchronises the stream
+    torch.cuda.synchronize(dev)
+    e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3, dev)
+    return e2e_ms, h2d, d2h
 
-    k_read, moved = algorithmic_bytes(wl, lens0.cpu().numpy())
-    peak, peak_kind = _peaks()
+
+def run_ours(args, rank, world, local_rank):
+    from paper_2605_23200_b200 import binding, build
+    import torch.distributed as dist
+
+    if rank == 0:
+        build.build()
+    dev = torch.device(f"cuda:{local_rank}")
+    torch.cuda.set_device(dev)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+        barrier()
+    binding.lib()
+    peaks = _peaks()
+    head_cfg = args.config if args.config is not None else HEADLINE_CFG
+    warmup = max(args.warmup, 3)
+
+    # ---- headline: first event of the headline configuration
+    b = Bench(head_cfg, dev, args.layers)
+    wl = b.wl
+    b.warm(warmup)
+    step = b.step
+    if args.graph:
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            b.step()
+        step = graph.replay
+        b.stream = torch.cuda.current_stream(dev)
+        for _ in range(3):
+            b.restore()
+            step()
+        b.comp.status()
+        torch.cuda.synchronize(dev)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    per_step = b.timed(args.steps, step)
+    barrier()
+    clocks = sampler.stop()
+    b.comp.status()
+    total_ms = max_over_ranks(float(sum(per_step)), dev)
+    launches = b.comp.last_launch_count * args.steps
+    kern_ms = b.kernel_times(min(args.steps, 10))
+    lens = b.lens0.cpu().numpy()
+    e2e = None
+    if not args.no_e2e:
+        n_e2e = min(args.steps, 50)
+        e2e_ms, h2d, d2h = e2e_loop(b, n_e2e)
+        e2e = {"value": world * n_e2e / (e2e_ms / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "steps": n_e2e,
+               "note": "uploads of step i+1 and the read-back of step i-1 overlap the kernels of step i (three buffer sets, three "
+                       "streams, at most two steps in flight); every step uploads all its inputs and its block table and lengths "
+                       "are read back and checked"}
     ms_per_step = total_ms / args.steps
-    dominant = max(kern_ms, key=kern_ms.get)
-    dom_bytes = moved if dominant == "gather" else k_read
-    dom_ms = kern_ms[dominant]
+    total_bytes = b.k_read + b.moved
     out = {
         "metric": METRIC, "value": world * args.steps / (total_ms / 1e3), "unit": UNIT, "n_gpus": world,
-        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "steps": args.steps, "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "dtype_detail": "bf16 K/V and queries, fp32 accumulation and scores, u64 fixed-point decisions",
         "data": "synthetic",
-        "config": {"workload": wl.name, "layers": wl.n_layers, "q_heads": wl.n_q_heads, "kv_heads": wl.n_kv_heads,
-                   "batch_per_gpu": wl.batch, "cache_tokens": wl.seq_len_max, "budget": wl.budget, "window": wl.window,
-                   "n_segments": wl.n_segments, "scorer": "tova" if wl.scorer_id == 0 else "keydiff",
-                   "l2": "inputs larger than L2 (K read per step %.2f GB)" % (k_read / 1e9),
-                   "parallelism": f"replica x{world}" if world > 1 else "single GPU",
-                   "launch": "one CUDA graph per step" if args.graph else "direct kernel launches"},
-        "effective_hbm_gbs": (k_read + moved) / (ms_per_step * 1e-3) / 1e9,
-        "effective_hbm_frac_of_8tbs": (k_read + moved) / (ms_per_step * 1e-3) / 8e12,
-        "effective_hbm_frac_of_measured": (k_read + moved) / (ms_per_step * 1e-3) / (peak * 1e9),
-        "algorithmic_bytes_per_step": k_read + moved,
+        "config": config_dict(wl),
+        "run": {"l2": "inputs larger than L2 (K read per step %.2f GB)" % (b.k_read / 1e9) if b.flush is None
+                      else "L2 flushed between timed steps (256 MB written)",
+                "parallelism": f"replica x{world}" if world > 1 else "single GPU",
+                "launch": "one CUDA graph per step" if args.graph else "direct kernel launches"},
+        "effective_hbm_gbs": total_bytes / (ms_per_step * 1e-3) / 1e9,
+        "effective_hbm_frac_of_8tbs": total_bytes / (ms_per_step * 1e-3) / 8e12,
+        "effective_hbm_frac_of_measured": total_bytes / (ms_per_step * 1e-3) / (peaks["hbm_gbs"] * 1e9),
+        "algorithmic_bytes_per_step": total_bytes,
         "gpu_launches": launches,
         "kernels_ms": kern_ms,
-        "roofline": {"kernel": dominant, "bound": "hbm", "achieved": dom_bytes / (dom_ms * 1e-3) / 1e9, "peak": peak,
-                     "peak_kind": peak_kind, "unit": "GB/s", "frac": dom_bytes / (dom_ms * 1e-3) / 1e9 / peak,
-                     "traffic": NCU_TRAFFIC_BYTES.get(wl.name, {}).get(dominant), "algorithmic_bytes_per_launch": dom_bytes,
-                     "note": "achieved = algorithmic bytes of the launch / mean CUDA-event duration of that kernel; "
-                             "frac is of the measured copy bandwidth"},
-        "e2e": None if e2e_ms is None else {"value": world * n_e2e / (e2e_ms / 1e3), "unit": UNIT,
-                                            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e,
-                                            "note": "uploads of step i+1 and the read-back of step i-1 overlap the kernels of step i (three buffer sets, three streams, at most two steps in flight); every step uploads all its inputs and its block table and lengths are read back and checked"},
+        "roofline": roofline_of(wl, kern_ms, b.k_read, b.moved, lens, peaks, NCU_TRAFFIC_BYTES.get(wl.name)),
+        "e2e": e2e,
         "clocks": clocks,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        out["cpu_baseline"] = cpu_baseline(wl, cache, dst_np, table0, lens0, budget_s=20.0)
+        out["cpu_baseline"] = cpu_baseline(wl, b.cache, b.dst_np, b.table0, b.lens0, budget_s=20.0)
+    steady_head = None
+    if not args.no_per_config and wl.steps > 1 and not args.layers:
+        steady_head = steady_state(b)
+    b.close()
+
+    # ---- all five configurations (rank 0's replica; every rank runs them so that the ranks stay in step)
+    if not args.no_per_config and args.config is None and not args.layers:
+        per = {}
+        for cid in range(5):
+            if cid == head_cfg:
+                e = {"workload": wl.name, "ms_per_step": ms_per_step, "steps_per_s": 1e3 / ms_per_step,
+                     "algorithmic_bytes_per_step": total_bytes, "effective_hbm_gbs": out["effective_hbm_gbs"],
+                     "effective_hbm_frac_of_8tbs": out["effective_hbm_frac_of_8tbs"], "kernels_ms": kern_ms,
+                     "roofline": out["roofline"], "launches_per_step": launches // args.steps, "note": "the headline measurement above"}
+                if steady_head:
+                    e["steady_state"] = steady_head
+                per[f"cfg{cid}"] = e
+                continue
+            bb, entry, _ = measure_config(cid, dev, min(args.steps, 10), 3, peaks)
+            bb.close()
+            per[f"cfg{cid}"] = entry
+        out["per_config"] = per
+    elif steady_head:
+        out["steady_state"] = steady_head
     if world > 1:
         dist.destroy_process_group()
     if rank == 0:
@@ -362,71 +558,124 @@ def cpu_baseline(wl, cache, dst_np, table0, lens0, budget_s):
     t0 = time.perf_counter()
     probe(1)
     unit_s = time.perf_counter() - t0
-    n = int(max(cores, min(len(units), budget_s * cores / max(unit_s, 1e-6))))
-    n = max(1, min(n, len(units)))
+    n = int(max(1, min(len(units), budget_s * cores / max(unit_s, 1e-6))))
+    if n >= cores:
+        n = n // cores * cores          # whole rounds of one unit per core
     sample = units[:n]
     run = _oracle_sample(wl, cache, dst_np, table0, lens0, sample)
     t0 = time.perf_counter()
-    run(cores)
+    run(min(cores, n))
     dt = time.perf_counter() - t0
-    return {"value": (n / len(units)) / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"first {n} of {len(units)} (layer, sequence, KV head) units, scaled by units; {dt:.1f} s wall"}
+    return {"value": (n / len(units)) / dt, "unit": UNIT, "cores": min(cores, n), "kind": "oracle",
+            "sample": f"first {n} of {len(units)} (layer, sequence, KV head) units, scaled by units; {dt:.1f} s wall "
+                      f"(one unit alone: {unit_s:.1f} s on one core)"}
 
 
 def run_reference(args, rank, world):
-    """Reference arm: the CPU oracle, unmodified, on the host cores, same metric and workload."""
+    """Reference arm: the CPU oracle, as it stands, on the host cores, same metric and workload.  One step is
+    a bounded sample of the workload's units (whole units: a unit is the smallest independent piece of the
+    path), scaled by units; a unit of the headline workload takes the oracle some twenty seconds on one core, so
+    the sample is one unit per core, the warm-up one step, and the number of timed steps is bounded."""
     if rank != 0:
         return
     from paper_2605_23200_b200 import inputs
-    wl = inputs.CONFIGS[args.config]
+    cfg_id = args.config if args.config is not None else HEADLINE_CFG
+    wl = inputs.CONFIGS[cfg_id]
     dev = "cuda:0" if torch.cuda.is_available() else "cpu"
-    cache = inputs.make_cache(wl, dev)
+    # only the sampled units' layers are needed on the host: build the cache with as few layers as the sample spans
+    cores = os.cpu_count() or 1
+    per_layer = wl.batch * wl.n_kv_heads
+    layers_needed = max(1, min(wl.layers_resident, -(-cores // per_layer)))
+    wl_small = wl.scaled(n_layers=layers_needed, resident_layers=0) if layers_needed < wl.layers_resident else wl
+    cache = inputs.make_cache(wl_small, dev)
     dst_np = inputs.alloc_dst_pages(cache)
     table0, lens0 = cache.block_table.clone(), cache.seq_lens.clone()
-    cores = os.cpu_count() or 1
-    units = _all_units(wl)
-    probe = _oracle_sample(wl, cache, dst_np, table0, lens0, units[:1])
+    units_all = len(_all_units(wl))
+    units = _all_units(wl_small)
+    probe = _oracle_sample(wl_small, cache, dst_np, table0, lens0, units[:1])
     t0 = time.perf_counter(); probe(1); unit_s = time.perf_counter() - t0
-    total_steps = args.steps + args.warmup
-    per_step_budget = 150.0 / max(total_steps, 1)
-    n = int(max(1, min(len(units), per_step_budget * cores / max(unit_s, 1e-6))))
-    run = _oracle_sample(wl, cache, dst_np, table0, lens0, units[:n])
-    for _ in range(args.warmup):
-        run(cores)
+    # A unit is the smallest independent piece of the path, so a step cannot be shorter than one unit's time on
+    # one core; the run is kept to a few minutes by timing at most as many steps as fit 200 s (never fewer than 3)
+    # after one warm-up step, and the line says how many were timed.
+    warmup = min(args.warmup, 1)
+    n = int(max(1, min(len(units), cores)))
+    steps = int(max(3, min(args.steps, 200.0 / max(unit_s, 1e-6))))
+    run = _oracle_sample(wl_small, cache, dst_np, table0, lens0, units[:n])
+    for _ in range(warmup):
+        run(min(cores, n))
     t0 = time.perf_counter()
-    for _ in range(args.steps):
-        run(cores)
+    for _ in range(steps):
+        run(min(cores, n))
     dt = time.perf_counter() - t0
-    value = args.steps * (n / len(units)) / dt
-    sample = f"each step = first {n} of {len(units)} units, scaled by units"
+    value = steps * (n / units_all) / dt
+    sample = (f"each step = first {n} of {units_all} units (whole units, one per core), scaled by units; one unit alone takes "
+              f"{unit_s:.1f} s on one core; {steps} of the {args.steps} requested steps timed after {warmup} warm-up step(s) "
+              f"so that the run ends within a few minutes")
     print(json.dumps({
-        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3 * (len(units) / n), "higher_is_better": True,
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
+        "steps_requested": args.steps, "warmup": warmup, "ms_per_step": dt / steps * 1e3 * (units_all / n), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "config": config_dict(wl),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": min(cores, n), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
+
+
+def run_plumbing(args, rank, world):
+    """CPU check of the multi-rank harness (no kernels, no GPU): gloo ranks meet at the barrier, each reports a
+    known duration, the maximum over ranks is taken and rank 0 prints the line.  Used by the tests."""
+    import torch.distributed as dist
+    if world > 1:
+        dist.init_process_group("gloo")
+    barrier()
+    ms = 10.0 * (rank + 1)
+    total = max_over_ranks(ms)
+    barrier()
+    if world > 1:
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps({"impl": "plumbing", "n_gpus": world, "ms_max_over_ranks": total, "scaling": "weak",
+                          "value": world * args.steps / (total / 1e3)}))
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def spawn_ranks(n):
+    """`--gpus N` without a launcher: run this script as N ranks under torch.distributed.run and pass its
+    output through."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(_free_port()), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=1)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference", "plumbing"])
+    ap.add_argument("--config", type=int, default=None, help="time this configuration only (default: headline + all five)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true")
     ap.add_argument("--graph", action="store_true", help="time the step replayed from a CUDA graph")
     ap.add_argument("--layers", type=int, default=0, help="profiling only: run a reduced layer count")
     args = ap.parse_args()
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1:
+        sys.exit(spawn_ranks(args.gpus))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        raise SystemExit(f"bench.py: --gpus {args.gpus} but the launcher started {world} rank(s)")
+    if args.impl == "plumbing":
+        run_plumbing(args, rank, world)
+        return
     if args.impl == "reference":
-        if args.steps > 20:
-            args.steps = 20 if "--steps" not in " ".join(sys.argv) else args.steps
         run_reference(args, rank, world)
         return
     if not torch.cuda.is_available():

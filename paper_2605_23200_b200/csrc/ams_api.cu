@@ -8,7 +8,7 @@
 namespace ams {
 
 struct Layout {
-    size_t status, eff_lens, seq_bad, scores, usage, logits, qctrl, cbuf, flags, n_seg, raw_cuts, seg_bounds, quotas, keep_idx, part, fin, total;
+    size_t status, eff_lens, seq_bad, scores, usage, logits, cbuf, n_seg, raw_cuts, seg_bounds, quotas, keep_idx, part, fin, total;
     int units, T_cap, seg_cap, n_slices, slice_len, rows_pad_cap;
 };
 
@@ -89,7 +89,6 @@ static Layout make_layout(const ams_config *c)
     // second per-token array: the usage when it is smoothed or comes from another scorer than the base scores
     y.usage = off;      off = align_up(off + ((c->pool_kernel > 1 || c->decoupled) ? U * T * 4 : 0), 256);
     y.cbuf = off;       off = align_up(off + U * T * 8, 256);
-    y.flags = off;      off = align_up(off + U * T, 256);
     y.n_seg = off;      off = align_up(off + U * 4, 256);
     y.raw_cuts = off;   off = align_up(off + U * (size_t)(c->max_segments + 1) * 4, 256);
     y.seg_bounds = off; off = align_up(off + U * (size_t)(y.seg_cap + 1) * 4, 256);
@@ -102,7 +101,6 @@ static Layout make_layout(const ams_config *c)
     // narrow query blocks keep their logits (rows_pad floats per token, at most 1/4 of the K bytes) so that
     // the usage pass need not read K again
     y.logits = off;     off = align_up(off + (y.rows_pad_cap <= 16 && c->max_window > 0 ? U * T * (size_t)y.rows_pad_cap * 4 : 0), 256);
-    y.qctrl = off;      off = align_up(off + (size_t)(4 + c->n_layers * c->max_batch) * 4, 256);
     y.total = off;
     return y;
 }
@@ -185,7 +183,6 @@ int ams_init_state(const ams_config *cfg, void *ema_state, void *workspace, size
     if (cudaMemsetAsync(workspace, 0, lay.scores, s) != cudaSuccess) return AMS_ERR_CUDA;
     if (cudaMemsetAsync((unsigned char *)workspace + lay.n_seg, 0, lay.raw_cuts - lay.n_seg, s) != cudaSuccess) return AMS_ERR_CUDA;
     if (cudaMemsetAsync((unsigned char *)workspace + lay.keep_idx, 0, lay.part - lay.keep_idx, s) != cudaSuccess) return AMS_ERR_CUDA;
-    if (cudaMemsetAsync((unsigned char *)workspace + lay.qctrl, 0, lay.total - lay.qctrl, s) != cudaSuccess) return AMS_ERR_CUDA;
     ams_state *st = new (std::nothrow) ams_state;
     if (!st) return AMS_ERR_INTERNAL;
     st->cfg = *cfg;
@@ -249,7 +246,7 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
         p.usage = ext_usage ? ext_usage : ext_scores;
     }
     float *usage_buf = (float *)(st->ws + y.usage);
-    p.cbuf = (u64 *)(st->ws + y.cbuf); p.flags = st->ws + y.flags;
+    p.cbuf = (u64 *)(st->ws + y.cbuf);
     p.n_seg = (int *)(st->ws + y.n_seg); p.seg_bounds = (int *)(st->ws + y.seg_bounds);
     p.quotas = (int *)(st->ws + y.quotas); p.keep_idx = (int *)(st->ws + y.keep_idx);
     p.raw_cuts = (int *)(st->ws + y.raw_cuts);
@@ -260,7 +257,6 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
     p.tc_tpc_min = tc_tiles_per_block_min(y.T_cap);
     p.tc_stages = p.rows_pad <= 256 ? 4 : 2; // even: each stage then belongs to one of the two MMA issuers
     p.status = (int *)(st->ws + y.status);
-    p.qctrl = (int *)(st->ws + y.qctrl);
     p.logits = (y.rows_pad_cap <= 16 && c.max_window > 0) ? (float *)(st->ws + y.logits) : nullptr;
 
     int rc = AMS_OK;
@@ -294,12 +290,7 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
         rc = launch_smooth_usage(p, p.usage, usage_buf, c.pool_kernel, ctx);
         p.usage = usage_buf;
     }
-    bool queued = false;
-    if (rc == AMS_OK) {
-        if (segsel_supported(p)) rc = launch_segsel(p, ctx);
-        else if (segment_cluster_supported(p)) { queued = segment_moves_rows(p); rc = launch_segment_select_cluster(p, ctx); }
-        else rc = launch_segment_select(p, ctx);
-    }
+    if (rc == AMS_OK) rc = segsel_supported(p) ? launch_segsel(p, ctx) : AMS_ERR_UNSUPPORTED;
     if (rc == AMS_OK && dbg) {
         // inspection copies are taken before the table is rewritten
         const size_t U = (size_t)p.L * p.B * p.H;
@@ -313,7 +304,7 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
         if (e != cudaSuccess) rc = AMS_ERR_CUDA;
         if (rc == AMS_OK && dbg->prev_kept && dbg->retained_iou) rc = launch_retained_iou(p, dbg->prev_kept, dbg->retained_iou, ctx);
     }
-    if (rc == AMS_OK) rc = launch_gather(p, ctx, queued);
+    if (rc == AMS_OK) rc = launch_gather(p, ctx);
     st->last_launches = ctx.launches;
     st->n_ev = ctx.n_ev;
     memcpy(st->ev_ids, ctx.ids, sizeof ctx.ids);

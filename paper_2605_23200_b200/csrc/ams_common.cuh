@@ -53,7 +53,6 @@ struct DevParams {
     int slice_len, n_slices, rows_pad;
     int tc_tpc_min, tc_stages;        // tensor-core scorer: least tiles per block, K stages in shared memory
     int tc_hpb;                       // tensor-core scorer: KV heads a block takes one after the other (set by its launcher)
-    int *qctrl;                       // work-queue counters of the one-block segmentation kernel, [4 + L * Bmax], zero between events
     float *logits;                    // narrow query blocks (rows_pad <= 16): scaled logits [units][T_cap][rows_pad], or null
     int *seq_bad;                     // [B]: set when a unit of the sequence reported a device-side error (its rows stay)
     int *status;                      // [4]: code, unit, a, b
@@ -232,14 +231,9 @@ bool tova_tc_supported(const DevParams &p);
 size_t tova_tc_smem_bytes(const DevParams &p);
 int launch_score_tova_tc(const DevParams &p, LaunchCtx &ctx);
 int launch_score_keydiff(const DevParams &p, LaunchCtx &ctx);
-int launch_segment_select(const DevParams &p, LaunchCtx &ctx);
-bool segsel_supported(const DevParams &p);   // the three-kernel form of Algorithm 1 steps 1-5
-int launch_segsel(const DevParams &p, LaunchCtx &ctx);
-bool segment_cluster_supported(const DevParams &p);
-bool segment_moves_rows(const DevParams &p); // the segmentation launch also starts the paged compaction
-int launch_segment_select_cluster(const DevParams &p, LaunchCtx &ctx);
-constexpr int kMoveRows = 512; // (token, head) rows of K and V per chunk of the paged compaction
-int launch_gather(const DevParams &p, LaunchCtx &ctx, bool queued); // queued: chunks below p.qctrl[1] are moved already
+bool segsel_supported(const DevParams &p);   // shared-memory need of the selection kernels fits (always, within the configuration limits)
+int launch_segsel(const DevParams &p, LaunchCtx &ctx); // Algorithm 1 steps 1-5: three kernels
+int launch_gather(const DevParams &p, LaunchCtx &ctx);
 int launch_smooth_usage(const DevParams &p, const float *src, float *dst, int k, LaunchCtx &ctx);
 // First kernel of an event: validates lengths and page ids, writes the effective lengths (lens_in: the caller's).
 int launch_prepare(const DevParams &p, const int *lens_in, int *eff_lens, LaunchCtx &ctx);

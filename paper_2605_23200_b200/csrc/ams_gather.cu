@@ -14,16 +14,10 @@ constexpr int kRowsPerBlock = kRowsPerIter * kUnroll;
 
 // Rows of one (layer, sequence) are numbered r = j * H + h, so that consecutive rows
 // are consecutive 256-byte pieces of the destination page.
-// queued: the chunks (kMoveRows rows each, in (layer, sequence) order) below p.qctrl[1] were moved by the
-// segmentation kernel already.
-__global__ void __launch_bounds__(kGatherThreads) k_gather(DevParams p, int queued)
+__global__ void __launch_bounds__(kGatherThreads) k_gather(DevParams p)
 {
-    wait_for_previous_kernel(); // kept positions and the count of chunks already moved
+    wait_for_previous_kernel(); // kept positions
     const int lb = blockIdx.y;
-    if (queued) {
-        const int chunks = (p.Tk * p.H + kMoveRows - 1) / kMoveRows;
-        if (lb * chunks + (int)(blockIdx.x * kRowsPerBlock) / kMoveRows < p.qctrl[1]) return;
-    }
     const int b = lb % p.B, l = lb / p.B;
     const int T = p.seq_lens[b];
     if (T <= p.Tk || T > p.T_cap || p.seq_bad[b]) return;
@@ -76,12 +70,11 @@ __global__ void k_table_update(DevParams p)
 
 } // namespace
 
-int launch_gather(const DevParams &p, LaunchCtx &ctx, bool queued)
+int launch_gather(const DevParams &p, LaunchCtx &ctx)
 {
-    static_assert(kMoveRows % kRowsPerBlock == 0, "a block of the gather kernel lies inside one chunk");
     const int n_rows = p.Tk * p.H;
     dim3 grid((n_rows + kRowsPerBlock - 1) / kRowsPerBlock, p.L * p.B);
-    if (launch_after(k_gather, grid, dim3(kGatherThreads), 0, ctx.s, p, queued ? 1 : 0) != cudaSuccess) return AMS_ERR_CUDA;
+    if (launch_after(k_gather, grid, dim3(kGatherThreads), 0, ctx.s, p) != cudaSuccess) return AMS_ERR_CUDA;
     ctx.mark(kKernGather);
     if (launch_after(k_table_update, dim3((unsigned)p.B), dim3(128), 0, ctx.s, p) != cudaSuccess) return AMS_ERR_CUDA;
     ctx.mark(kKernTable);

@@ -324,19 +324,6 @@ __global__ void __launch_bounds__(1024) k_segment_select(DevParams p)
     }
 }
 
-int launch_segment_select(const DevParams &p, LaunchCtx &ctx)
-{
-    const int units = p.L * p.B * p.H;
-    const int nthreads = 1024;
-    const size_t dyn = (size_t)p.seg_cap * 8 + (size_t)(4 * p.seg_cap + 1) * 4 + (size_t)3 * (p.S + 1) * 4 +
-                       (size_t)(nthreads / 32) * (256 + 4) * 4 + 64;
-    static SmemGrant grant;
-    if (!grant_dynamic_smem(k_segment_select, dyn, grant)) return AMS_ERR_CUDA;
-    k_segment_select<<<units, nthreads, dyn, ctx.s>>>(p);
-    ctx.mark(kKernSegmentSelect);
-    return cudaGetLastError() == cudaSuccess ? AMS_OK : AMS_ERR_CUDA;
-}
-
 } // namespace ams
 
 // ---------------------------------------------------------------------------------------

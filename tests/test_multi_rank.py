@@ -58,3 +58,23 @@ def test_algorithmic_bytes_match_the_definition():
     wl = inputs.CONFIGS[2]
     k_read, moved = bench.algorithmic_bytes(wl, [4096, 9000])       # the first sequence is skipped
     assert k_read == 28 * 4 * 9000 * 256 and moved == 28 * 4 * 4096 * 1024
+
+
+def test_bench_gpus_flag_spawns_that_many_ranks():
+    """`bench.py --gpus 2` without a launcher starts two ranks itself (torch.distributed.run on 127.0.0.1);
+    with the CPU plumbing arm they meet over gloo, the slowest rank sets the time and one line is printed.
+    A launcher that disagrees with --gpus is refused."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "plumbing", "--steps", "7"],
+                         capture_output=True, text=True, timeout=300, env=env)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["ms_max_over_ranks"] == 20.0 and abs(line["value"] - 2 * 7 / 0.020) < 1e-6
+    env2 = dict(env, WORLD_SIZE="3", RANK="0", LOCAL_RANK="0")
+    bad = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "plumbing"],
+                         capture_output=True, text=True, timeout=120, env=env2)
+    assert bad.returncode != 0 and "--gpus 2" in (bad.stderr + bad.stdout)
