@@ -34,7 +34,6 @@ constexpr int kSelThreads = 256;
 constexpr int kSelWarps = kSelThreads / 32;
 constexpr int kRegKeys = 32;                // keys a thread can hold: segments up to kSelThreads * kRegKeys in registers
 constexpr int kListCap = 1024;              // backfill candidates kept in shared memory
-constexpr int kListPer = kListCap / kSelThreads;
 
 struct UnitId { int l, b, h; };
 __device__ __forceinline__ UnitId unit_of(const DevParams &p, int uid)
@@ -89,6 +88,25 @@ __device__ __forceinline__ void walk4x2(const float *row_a, const float *row_b, 
     }
 }
 
+// Block-wide sum of doubles that are integers below 2^53 (exact, hence independent of the order).
+__device__ __forceinline__ double block_sum_exact_f64(double v, u64 *scratch)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();
+    if (lane == 0) scratch[warp] = (u64)__double_as_longlong(v);
+    __syncthreads();
+    if (warp == 0) {
+        double x = lane < nw ? __longlong_as_double((long long)scratch[lane]) : 0.0;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+        if (lane == 0) scratch[32] = (u64)__double_as_longlong(x);
+    }
+    __syncthreads();
+    return __longlong_as_double((long long)scratch[32]);
+}
+
 // raw_cuts: [units][S + 1] cut positions of the mass quantiles (entry k: boundary after the token that
 // reaches k / S; T where no token before the last one does).
 __global__ void __launch_bounds__(kScanThreads) k_mass_scan(DevParams p)
@@ -123,20 +141,23 @@ __global__ void __launch_bounds__(kScanThreads) k_mass_scan(DevParams p)
     });
     wmax = block_max_f32(wmax, scratch);
     const int ew = fix_exponent(wmax);
-    // ---- SA = sum of the images
-    u64 sa = 0;
+    // ---- SA = sum of the images A_t = floor(w_t 2^(36 - ew)), held as doubles (integers below 2^53: exact)
+    const double scale_w = fix_scale_of(ew);
+    double sa = 0.0;
     walk4(u, T4, [&](int t, float4 v) {
         const float w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-        for (int i = 0; i < 4; ++i) if (t + i < T) sa += to_fixed_bits(weight_of(w[i], p.eps), ew);
+        for (int i = 0; i < 4; ++i)
+            if (t + i < T) sa = __dadd_rn(sa, __dmul_rn((double)fixed_trunc(weight_of(w[i], p.eps), ew), scale_w));
     });
-    const u64 SA = block_sum_u64(sa, scratch);
-    const double inv_sa = __ddiv_rn(1.0, (double)SA); // normalisations multiply by the rounded reciprocal
+    const double SA = block_sum_exact_f64(sa, scratch);
+    const double inv_sa = __ddiv_rn(1.0, SA);          // normalisations multiply by the rounded reciprocal
+    const double inv_sa_w = __dmul_rn(inv_sa, scale_w); // A_t / SA = trunc(w_t) * (2^(36 - ew) / SA): the scaling is exact
 
     // ---- EMA credit: c <- lambda c + (1 - lambda) m, updated in place (the block-wide reductions that follow
     //      make every thread's writes visible to the others before anybody reads them back)
     int ec = 0;
-    double inv_sc = 0.0;
+    double inv_sc_c = 0.0; // 2^(36 - ec) / SC
     bool have_credit = false;
     if (ema_on) {
         const float oml = __fsub_rn(1.0f, p.lambda);
@@ -147,7 +168,7 @@ __global__ void __launch_bounds__(kScanThreads) k_mass_scan(DevParams p)
             float m[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                m[i] = __double2float_rn(__dmul_rn(u52_to_double(to_fixed_bits(weight_of(w[i], p.eps), ew)), inv_sa));
+                m[i] = __double2float_rn(__dmul_rn((double)fixed_trunc(weight_of(w[i], p.eps), ew), inv_sa_w));
                 if (t + i < T) {
                     c[i] = __fadd_rn(__fmul_rn(p.lambda, c[i]), __fmul_rn(oml, m[i]));
                     cmax = fmaxf(cmax, c[i]);
@@ -163,18 +184,21 @@ __global__ void __launch_bounds__(kScanThreads) k_mass_scan(DevParams p)
             }
         });
         cmax = block_max_f32(cmax, scratch);
-        u64 scsum = 0;
+        double scsum = 0.0;
+        double scale_c = 0.0;
         if (cmax > 0.0f) {
             ec = fix_exponent(cmax);
+            scale_c = fix_scale_of(ec);
             walk4(credit, T4, [&](int t, float4 cv) {
                 const float c[4] = {cv.x, cv.y, cv.z, cv.w};
 #pragma unroll
-                for (int i = 0; i < 4; ++i) if (t + i < T) scsum += to_fixed_bits(c[i], ec);
+                for (int i = 0; i < 4; ++i)
+                    if (t + i < T) scsum = __dadd_rn(scsum, __dmul_rn((double)fixed_trunc(c[i], ec), scale_c));
             });
         }
-        const u64 SC = block_sum_u64(scsum, scratch);
-        have_credit = SC > 0;
-        if (have_credit) inv_sc = __ddiv_rn(1.0, (double)SC);
+        const double SC = block_sum_exact_f64(scsum, scratch);
+        have_credit = SC > 0.0;
+        if (have_credit) inv_sc_c = __dmul_rn(__ddiv_rn(1.0, SC), scale_c);
     }
 
     // ---- history-aware integer mass Hm_t = floor((beta m + (1 - beta) normalize(c)) 2^36) and its inclusive
@@ -214,10 +238,10 @@ __global__ void __launch_bounds__(kScanThreads) k_mass_scan(DevParams p)
                 u64 h = 0;
                 m[i] = 0.0f;
                 if (t + i < T) {
-                    const double r = __dmul_rn(u52_to_double(to_fixed_bits(weight_of(w[i], p.eps), ew)), inv_sa);
+                    const double r = __dmul_rn((double)fixed_trunc(weight_of(w[i], p.eps), ew), inv_sa_w);
                     if (ema_on) {
                         double hist = 0.0;
-                        if (have_credit) hist = __dmul_rn(omb, __dmul_rn(u52_to_double(to_fixed_bits(c[i], ec)), inv_sc));
+                        if (have_credit) hist = __dmul_rn(omb, __dmul_rn((double)fixed_trunc(c[i], ec), inv_sc_c));
                         h = floor_to_u64(__dmul_rn(__dadd_rn(__dmul_rn(bd, r), hist), two_f));
                     } else {
                         m[i] = __double2float_rn(r);
@@ -505,6 +529,8 @@ struct SelShared {
     u64 scratch[40];
     int wc[2][32];   // per-warp counts of even / odd search rounds
     int n_list;
+    unsigned bound;
+    unsigned tmax[kSelThreads];
 };
 
 // Sum of one count per thread over the block with one barrier per call: counts of consecutive calls land in
@@ -800,14 +826,27 @@ __global__ void __launch_bounds__(kSelThreads, 4) k_select_compact(DevParams p)
                 }
             };
             unsigned tmax = 0;
-            int have = 0;
-            walk([&](int, unsigned key) { tmax = max(tmax, key); have = 1; });
-            unsigned M = 0;
-            for (int bit = 31; bit >= 0; --bit) {
-                const unsigned X = M | (1u << bit);
-                const int tot = block_count(have && tmax >= X, round++, sh);
-                if (tot >= r_fill) M = X;
+            walk([&](int, unsigned key) { tmax = max(tmax, key); });
+            // r-th largest of the per-thread maxima, found by one warp (a maximum of 0 counts for nothing: a thread
+            // without candidates, or with NaN scores only, which then all qualify below)
+            sh.tmax[tid] = tmax;
+            __syncthreads();
+            if (warp == 0) {
+                unsigned tv[kSelThreads / 32];
+#pragma unroll
+                for (int j = 0; j < kSelThreads / 32; ++j) tv[j] = sh.tmax[j * 32 + lane];
+                unsigned M = 0;
+                for (int bit = 31; bit >= 0; --bit) {
+                    const unsigned X = M | (1u << bit);
+                    int c = 0;
+#pragma unroll
+                    for (int j = 0; j < kSelThreads / 32; ++j) c += tv[j] >= X;
+                    if (__reduce_add_sync(0xffffffffu, c) >= r_fill) M = X;
+                }
+                if (lane == 0) sh.bound = M;
             }
+            __syncthreads();
+            const unsigned M = sh.bound;
             walk([&](int t, unsigned key) {
                 if (key >= M) {
                     const int at = atomicAdd(&sh.n_list, 1);
@@ -817,45 +856,35 @@ __global__ void __launch_bounds__(kSelThreads, 4) k_select_compact(DevParams p)
             __syncthreads();
             const int n_list = sh.n_list;
             if (n_list <= kListCap) {
-                // the list is in arrival order: ties are ranked by position, not by list index
-                unsigned k4[kListPer], pos4[kListPer];
-                unsigned elig = 0;
-#pragma unroll
-                for (int j = 0; j < kListPer; ++j) {
-                    const int i = j * kSelThreads + tid;
-                    k4[j] = 0u; pos4[j] = 0u;
-                    if (i < n_list) { const uint2 v = list[i]; k4[j] = v.x; pos4[j] = v.y; elig |= 1u << j; }
-                }
-                unsigned P = 0;
-                bool exact = false;
-                for (int bit = 31; bit >= 0; --bit) {
-                    const unsigned X = P | (1u << bit);
-                    int c = 0;
-#pragma unroll
-                    for (int j = 0; j < kListPer; ++j) c += k4[j] >= X;
-                    const int tot = block_count(c, round++, sh);
-                    if (tot >= r_fill) { P = X; if (tot == r_fill) { exact = true; break; } }
-                }
-                unsigned P2 = 0;
-                if (!exact) {
-                    int c = 0;
-#pragma unroll
-                    for (int j = 0; j < kListPer; ++j) c += ((elig >> j) & 1u) && k4[j] > P;
-                    const int take = r_fill - block_count(c, round++, sh);
-                    for (int bit = 31 - __clz(T); bit >= 0; --bit) {
-                        const unsigned X = P2 | (1u << bit);
-                        int c2 = 0;
-#pragma unroll
-                        for (int j = 0; j < kListPer; ++j)
-                            c2 += ((elig >> j) & 1u) && k4[j] == P && (unsigned)T - pos4[j] >= X;
-                        const int tot = block_count(c2, round++, sh);
-                        if (tot >= take) { P2 = X; if (tot == take) break; }
+                // Top r_fill of the list by (key desc, position asc), one warp, entries strided over the lanes.  The
+                // list is in arrival order, so ties are ranked by position, not by list index.
+                if (warp == 0) {
+                    auto count = [&](auto pred) {
+                        int c = 0;
+                        for (int i = lane; i < n_list; i += 32) c += pred(list[i]);
+                        return __reduce_add_sync(0xffffffffu, c);
+                    };
+                    unsigned P = 0;
+                    bool exact = false;
+                    for (int bit = 31; bit >= 0; --bit) {
+                        const unsigned X = P | (1u << bit);
+                        const int tot = count([&](uint2 v) { return v.x >= X; });
+                        if (tot >= r_fill) { P = X; if (tot == r_fill) { exact = true; break; } }
+                    }
+                    unsigned P2 = 0;
+                    if (!exact) {
+                        const int take = r_fill - count([&](uint2 v) { return v.x > P; });
+                        for (int bit = 31 - __clz(T); bit >= 0; --bit) {
+                            const unsigned X = P2 | (1u << bit);
+                            const int tot = count([&](uint2 v) { return v.x == P && (unsigned)T - v.y >= X; });
+                            if (tot >= take) { P2 = X; if (tot == take) break; }
+                        }
+                    }
+                    for (int i = lane; i < n_list; i += 32) {
+                        const uint2 v = list[i];
+                        if (v.x > P || (v.x == P && (exact || (unsigned)T - v.y >= P2))) raise((int)v.y);
                     }
                 }
-#pragma unroll
-                for (int j = 0; j < kListPer; ++j)
-                    if (((elig >> j) & 1u) && (k4[j] > P || (k4[j] == P && (exact || (unsigned)T - pos4[j] >= P2))))
-                        raise((int)pos4[j]);
             } else {
                 block_select_stream(T, r_fill, sh, round, key_at, unflagged, raise);
             }

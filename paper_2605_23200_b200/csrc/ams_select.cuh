@@ -185,6 +185,25 @@ __device__ __forceinline__ u64 to_fixed_bits(float x, int e)
     return sh >= 0 ? (m << sh) : (sh > -24 ? (m >> (-sh)) : 0ull);
 }
 
+// The fixed-point image A = floor(x * 2^(kFixBits - e)) (0 <= x < 2^e) equals trunc(x) * 2^(kFixBits - e), where
+// trunc(x) is x with the mantissa bits below the image's last bit cleared: x = m * 2^(E - 23), and the image
+// drops the lowest n = e - 13 - E bits of m when that is positive (all 24 of them from n = 24 on).  So the
+// image is available as a double with one conversion and one exact multiplication by a power of two, and
+// sums of images (integers below 2^53) can be added in fp64 in any order.
+__device__ __forceinline__ float fixed_trunc(float x, int e)
+{
+    const unsigned b = __float_as_uint(x);
+    const int ef = max((int)((b >> 23) & 0xffu), 1); // subnormals share the scale of the smallest normal exponent
+    const int n = e - (kFixBits - 23) - (ef - 127);
+    return n <= 0 ? x : (n >= 24 ? 0.0f : __uint_as_float(b & (0xffffffffu << n)));
+}
+
+// 2^(kFixBits - e) as a double (e = fix_exponent of a positive fp32, so the result is a normal double).
+__device__ __forceinline__ double fix_scale_of(int e)
+{
+    return __longlong_as_double((long long)(1023 + kFixBits - e) << 52);
+}
+
 // (double)a for an integer a < 2^52, exact.
 __device__ __forceinline__ double u52_to_double(u64 a)
 {
