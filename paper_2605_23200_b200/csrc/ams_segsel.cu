@@ -30,9 +30,6 @@ namespace {
 
 constexpr int kScanThreads = 512;
 constexpr int kScanVec = 8;                 // tokens per thread and round of the scan pass
-constexpr int kSelThreads = 256;
-constexpr int kSelWarps = kSelThreads / 32;
-constexpr int kRegKeys = 32;                // keys a thread can hold: segments up to kSelThreads * kRegKeys in registers
 constexpr int kListCap = 1024;              // backfill candidates kept in shared memory
 
 struct UnitId { int l, b, h; };
@@ -143,12 +140,13 @@ __global__ void __launch_bounds__(kScanThreads) k_mass_scan(DevParams p)
     const int ew = fix_exponent(wmax);
     // ---- SA = sum of the images A_t = floor(w_t 2^(36 - ew)), held as doubles (integers below 2^53: exact)
     const double scale_w = fix_scale_of(ew);
+    const float cut_w = fixed_trunc_threshold(ew); // weights below it lose their bits under the image's last one
     double sa = 0.0;
     walk4(u, T4, [&](int t, float4 v) {
         const float w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-            if (t + i < T) sa = __dadd_rn(sa, __dmul_rn((double)fixed_trunc(weight_of(w[i], p.eps), ew), scale_w));
+            if (t + i < T) sa = __dadd_rn(sa, __dmul_rn((double)fixed_trunc_by_add(weight_of(w[i], p.eps), cut_w), scale_w));
     });
     const double SA = block_sum_exact_f64(sa, scratch);
     const double inv_sa = __ddiv_rn(1.0, SA);          // normalisations multiply by the rounded reciprocal
@@ -157,6 +155,7 @@ __global__ void __launch_bounds__(kScanThreads) k_mass_scan(DevParams p)
     // ---- EMA credit: c <- lambda c + (1 - lambda) m, updated in place (the block-wide reductions that follow
     //      make every thread's writes visible to the others before anybody reads them back)
     int ec = 0;
+    float cut_c = 0.0f;
     double inv_sc_c = 0.0; // 2^(36 - ec) / SC
     bool have_credit = false;
     if (ema_on) {
@@ -168,7 +167,7 @@ __global__ void __launch_bounds__(kScanThreads) k_mass_scan(DevParams p)
             float m[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                m[i] = __double2float_rn(__dmul_rn((double)fixed_trunc(weight_of(w[i], p.eps), ew), inv_sa_w));
+                m[i] = __double2float_rn(__dmul_rn((double)fixed_trunc_by_add(weight_of(w[i], p.eps), cut_w), inv_sa_w));
                 if (t + i < T) {
                     c[i] = __fadd_rn(__fmul_rn(p.lambda, c[i]), __fmul_rn(oml, m[i]));
                     cmax = fmaxf(cmax, c[i]);
@@ -189,11 +188,12 @@ __global__ void __launch_bounds__(kScanThreads) k_mass_scan(DevParams p)
         if (cmax > 0.0f) {
             ec = fix_exponent(cmax);
             scale_c = fix_scale_of(ec);
+            cut_c = fixed_trunc_threshold(ec);
             walk4(credit, T4, [&](int t, float4 cv) {
                 const float c[4] = {cv.x, cv.y, cv.z, cv.w};
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
-                    if (t + i < T) scsum = __dadd_rn(scsum, __dmul_rn((double)fixed_trunc(c[i], ec), scale_c));
+                    if (t + i < T) scsum = __dadd_rn(scsum, __dmul_rn((double)fixed_trunc_by_add(c[i], cut_c), scale_c));
             });
         }
         const double SC = block_sum_exact_f64(scsum, scratch);
@@ -238,10 +238,10 @@ __global__ void __launch_bounds__(kScanThreads) k_mass_scan(DevParams p)
                 u64 h = 0;
                 m[i] = 0.0f;
                 if (t + i < T) {
-                    const double r = __dmul_rn((double)fixed_trunc(weight_of(w[i], p.eps), ew), inv_sa_w);
+                    const double r = __dmul_rn((double)fixed_trunc_by_add(weight_of(w[i], p.eps), cut_w), inv_sa_w);
                     if (ema_on) {
                         double hist = 0.0;
-                        if (have_credit) hist = __dmul_rn(omb, __dmul_rn((double)fixed_trunc(c[i], ec), inv_sc_c));
+                        if (have_credit) hist = __dmul_rn(omb, __dmul_rn((double)fixed_trunc_by_add(c[i], cut_c), inv_sc_c));
                         h = floor_to_u64(__dmul_rn(__dadd_rn(__dmul_rn(bd, r), hist), two_f));
                     } else {
                         m[i] = __double2float_rn(r);
@@ -530,12 +530,13 @@ struct SelShared {
     int wc[2][32];   // per-warp counts of even / odd search rounds
     int n_list;
     unsigned bound;
-    unsigned tmax[kSelThreads];
+    unsigned tmax[512];
 };
 
 // Sum of one count per thread over the block with one barrier per call: counts of consecutive calls land in
 // alternating tables, so a table is rewritten only after every thread has passed the barrier that follows
 // its last read.
+template <int NT>
 __device__ __forceinline__ int block_count(int c, int round, SelShared &sh)
 {
     const int lane = threadIdx.x & 31;
@@ -543,7 +544,7 @@ __device__ __forceinline__ int block_count(int c, int round, SelShared &sh)
     int *mine = sh.wc[round & 1];
     if (lane == 0) mine[threadIdx.x >> 5] = c;
     __syncthreads();
-    const int v = lane < kSelWarps ? mine[lane] : 0;
+    const int v = lane < NT / 32 ? mine[lane] : 0;
     return __reduce_add_sync(0xffffffffu, v);
 }
 
@@ -561,15 +562,20 @@ __device__ __forceinline__ void mask_or_ballot(unsigned *mask, int t0, unsigned 
 // found bit by bit from the top (one warp-wide count per bit), stopping as soon as exactly q keys lie at or
 // above the prefix; of the keys equal to the threshold the first ones in position order are taken.
 template <int KPL>
-__device__ __forceinline__ void warp_segment(const float *g, unsigned *mask, int a, int e, int q)
+__device__ __forceinline__ void warp_load_keys(const float *g, int a, int e, unsigned (&k)[KPL])
 {
     const int lane = threadIdx.x & 31;
-    unsigned k[KPL];
 #pragma unroll
     for (int j = 0; j < KPL; ++j) {
         const int t = a + j * 32 + lane;
         k[j] = t < e ? score_key(g[t]) : 0u; // a key of 0 is never counted (X >= 1); real zeros are handled as ties of P = 0
     }
+}
+
+template <int KPL>
+__device__ __forceinline__ void warp_segment(const unsigned (&k)[KPL], unsigned *mask, int a, int e, int q)
+{
+    const int lane = threadIdx.x & 31;
     unsigned P = 0;
     bool exact = false;
     for (int bit = 31; bit >= 0; --bit) {
@@ -609,10 +615,10 @@ __device__ __forceinline__ void warp_segment(const float *g, unsigned *mask, int
 }
 
 // Top-q of the `n` items of a block-wide set, at most KPT per thread, item j of thread tid being number
-// j * kSelThreads + tid (numbers ascend with position).  key_of(i) gives the score key, ok(i) whether the item
+// j * NT + tid (numbers ascend with position).  key_of(i) gives the score key, ok(i) whether the item
 // takes part; keep(i) is called for every winner.  First the key bits, then (if more than q items lie at or
 // above the q-th key) the item numbers of the tied items, smaller first.
-template <int KPT, typename KeyOf, typename Ok, typename Keep>
+template <int NT, int KPT, typename KeyOf, typename Ok, typename Keep>
 __device__ __forceinline__ void block_select_reg(int n, int q, SelShared &sh, int &round, KeyOf key_of, Ok ok, Keep keep)
 {
     const int tid = threadIdx.x;
@@ -620,7 +626,7 @@ __device__ __forceinline__ void block_select_reg(int n, int q, SelShared &sh, in
     unsigned elig = 0;
 #pragma unroll
     for (int j = 0; j < KPT; ++j) {
-        const int i = j * kSelThreads + tid;
+        const int i = j * NT + tid;
         k[j] = 0u;
         if (i < n && ok(i)) { elig |= 1u << j; k[j] = key_of(i); }
     }
@@ -631,7 +637,7 @@ __device__ __forceinline__ void block_select_reg(int n, int q, SelShared &sh, in
         int c = 0;
 #pragma unroll
         for (int j = 0; j < KPT; ++j) c += k[j] >= X;
-        const int tot = block_count(c, round++, sh);
+        const int tot = block_count<NT>(c, round++, sh);
         if (tot >= q) {
             P = X;
             if (tot == q) { exact = true; break; }
@@ -644,12 +650,12 @@ __device__ __forceinline__ void block_select_reg(int n, int q, SelShared &sh, in
     if (!exact) {
         // ties at the threshold: the first (q - #above) of them by item number.  Search the item-number image
         // n - i (larger = earlier), unique per item, so the count ends exactly.
-        const int above = block_count(__popc(win), round++, sh);
+        const int above = block_count<NT>(__popc(win), round++, sh);
         const int take = q - above;
         unsigned tie = 0;
 #pragma unroll
         for (int j = 0; j < KPT; ++j) {
-            const int i = j * kSelThreads + tid;
+            const int i = j * NT + tid;
             const bool is_tie = ((elig >> j) & 1u) && k[j] == P;
             if (is_tie) tie |= 1u << j;
             k[j] = is_tie ? (unsigned)(n - i) : 0u;
@@ -660,7 +666,7 @@ __device__ __forceinline__ void block_select_reg(int n, int q, SelShared &sh, in
             int c = 0;
 #pragma unroll
             for (int j = 0; j < KPT; ++j) c += k[j] >= X;
-            const int tot = block_count(c, round++, sh);
+            const int tot = block_count<NT>(c, round++, sh);
             if (tot >= take) {
                 P2 = X;
                 if (tot == take) break;
@@ -672,11 +678,11 @@ __device__ __forceinline__ void block_select_reg(int n, int q, SelShared &sh, in
     }
 #pragma unroll
     for (int j = 0; j < KPT; ++j)
-        if ((win >> j) & 1u) keep(j * kSelThreads + tid);
+        if ((win >> j) & 1u) keep(j * NT + tid);
 }
 
 // The same selection for sets too large for registers: every round walks the items again (scores from L2).
-template <typename KeyOf, typename Ok, typename Keep>
+template <int NT, typename KeyOf, typename Ok, typename Keep>
 __device__ void block_select_stream(int n, int q, SelShared &sh, int &round, KeyOf key_of, Ok ok, Keep keep)
 {
     const int tid = threadIdx.x;
@@ -685,8 +691,8 @@ __device__ void block_select_stream(int n, int q, SelShared &sh, int &round, Key
     for (int bit = 31; bit >= 0; --bit) {
         const unsigned X = P | (1u << bit);
         int c = 0;
-        for (int i = tid; i < n; i += kSelThreads) c += ok(i) && key_of(i) >= X;
-        const int tot = block_count(c, round++, sh);
+        for (int i = tid; i < n; i += NT) c += ok(i) && key_of(i) >= X;
+        const int tot = block_count<NT>(c, round++, sh);
         if (tot >= q) {
             P = X;
             if (tot == q) { exact = true; break; }
@@ -695,37 +701,38 @@ __device__ void block_select_stream(int n, int q, SelShared &sh, int &round, Key
     unsigned P2 = 0;
     if (!exact) {
         int c = 0;
-        for (int i = tid; i < n; i += kSelThreads) c += ok(i) && key_of(i) > P;
-        const int take = q - block_count(c, round++, sh);
+        for (int i = tid; i < n; i += NT) c += ok(i) && key_of(i) > P;
+        const int take = q - block_count<NT>(c, round++, sh);
         for (int bit = 31 - __clz(n); bit >= 0; --bit) {
             const unsigned X = P2 | (1u << bit);
             int c2 = 0;
-            for (int i = tid; i < n; i += kSelThreads) c2 += ok(i) && key_of(i) == P && (unsigned)(n - i) >= X;
-            const int tot = block_count(c2, round++, sh);
+            for (int i = tid; i < n; i += NT) c2 += ok(i) && key_of(i) == P && (unsigned)(n - i) >= X;
+            const int tot = block_count<NT>(c2, round++, sh);
             if (tot >= take) {
                 P2 = X;
                 if (tot == take) break;
             }
         }
     }
-    for (int i = tid; i < n; i += kSelThreads) {
+    for (int i = tid; i < n; i += NT) {
         if (!ok(i)) continue;
         const unsigned key = key_of(i);
         if (key > P || (key == P && (exact || (unsigned)(n - i) >= P2))) keep(i);
     }
 }
 
-template <typename KeyOf, typename Ok, typename Keep>
+template <int NT, typename KeyOf, typename Ok, typename Keep>
 __device__ __forceinline__ void block_select(int n, int q, SelShared &sh, int &round, KeyOf key_of, Ok ok, Keep keep)
 {
-    if (n <= kSelThreads * 4) block_select_reg<4>(n, q, sh, round, key_of, ok, keep);
-    else if (n <= kSelThreads * 8) block_select_reg<8>(n, q, sh, round, key_of, ok, keep);
-    else if (n <= kSelThreads * 16) block_select_reg<16>(n, q, sh, round, key_of, ok, keep);
-    else if (n <= kSelThreads * kRegKeys) block_select_reg<kRegKeys>(n, q, sh, round, key_of, ok, keep);
-    else block_select_stream(n, q, sh, round, key_of, ok, keep);
+    if (n <= NT * 4) block_select_reg<NT, 4>(n, q, sh, round, key_of, ok, keep);
+    else if (n <= NT * 8) block_select_reg<NT, 8>(n, q, sh, round, key_of, ok, keep);
+    else if (n <= NT * 16) block_select_reg<NT, 16>(n, q, sh, round, key_of, ok, keep);
+    else if (NT <= 256 && n <= NT * 32) block_select_reg<NT, NT <= 256 ? 32 : 16>(n, q, sh, round, key_of, ok, keep);
+    else block_select_stream<NT>(n, q, sh, round, key_of, ok, keep);
 }
 
-__global__ void __launch_bounds__(kSelThreads, 4) k_select_compact(DevParams p)
+template <int NT>
+__global__ void __launch_bounds__(NT, 1024 / NT) k_select_compact(DevParams p)
 {
     extern __shared__ __align__(16) unsigned char dyn[];
     __shared__ SelShared sh;
@@ -748,33 +755,59 @@ __global__ void __launch_bounds__(kSelThreads, 4) k_select_compact(DevParams p)
     wait_for_previous_kernel(); // segments and quotas
     const int n_seg = p.n_seg[uid];
     if (n_seg < 0) return; // reported by the previous kernel
-    for (int i = tid; i <= n_words; i += kSelThreads) mask[i] = 0u;
-    for (int i = tid; i < n_seg; i += kSelThreads) {
+    for (int i = tid; i <= n_words; i += NT) mask[i] = 0u;
+    for (int i = tid; i < n_seg; i += NT) {
         bounds[i] = p.seg_bounds[(size_t)uid * (sc + 1) + i];
         quota[i] = p.quotas[(size_t)uid * sc + i];
     }
     if (tid == 0) { bounds[n_seg] = T; sh.n_list = 0; }
     __syncthreads();
 
-    // ---- per-segment top-q_i by (score desc, position asc): a warp per segment of at most 1024 tokens
+    // ---- per-segment top-q_i by (score desc, position asc): a warp per segment of at most 1024 tokens.  The keys of
+    //      the warp's next segment (the common case of at most 256 tokens) are fetched before the current one is
+    //      searched, so that their latency is hidden behind the search.
     bool any_long = false;
-    for (int s = warp; s < n_seg; s += kSelWarps) {
-        const int a = bounds[s], e = bounds[s + 1], q = quota[s], L = e - a;
-        if (q <= 0) continue;
-        if (q >= L) {
-            for (int t0 = a; t0 < e; t0 += 32) mask_or_ballot(mask, t0, __ballot_sync(0xffffffffu, t0 + lane < e));
-        } else if (L <= 128) warp_segment<4>(g, mask, a, e, q);
-        else if (L <= 256) warp_segment<8>(g, mask, a, e, q);
-        else if (L <= 512) warp_segment<16>(g, mask, a, e, q);
-        else if (L <= 1024) warp_segment<32>(g, mask, a, e, q);
-        else any_long = true;
+    {
+        auto searched = [&](int sg) { // a segment that needs a search and fits eight keys per lane
+            const int L = bounds[sg + 1] - bounds[sg], q = quota[sg];
+            return q > 0 && q < L && L <= 256;
+        };
+        unsigned kn[8];
+        bool have_next = false;
+        if (warp < n_seg && searched(warp)) { warp_load_keys<8>(g, bounds[warp], bounds[warp + 1], kn); have_next = true; }
+        for (int sg = warp; sg < n_seg; sg += (NT / 32)) {
+            const int a = bounds[sg], e = bounds[sg + 1], q = quota[sg], L = e - a;
+            unsigned kc[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) kc[j] = kn[j];
+            const bool have = have_next;
+            const int nx = sg + (NT / 32);
+            have_next = nx < n_seg && searched(nx);
+            if (have_next) warp_load_keys<8>(g, bounds[nx], bounds[nx + 1], kn);
+            if (q <= 0) continue;
+            if (q >= L) {
+                for (int t0 = a; t0 < e; t0 += 32) mask_or_ballot(mask, t0, __ballot_sync(0xffffffffu, t0 + lane < e));
+            } else if (have) {
+                warp_segment<8>(kc, mask, a, e, q);
+            } else if (L <= 512) {
+                unsigned k16[16];
+                warp_load_keys<16>(g, a, e, k16);
+                warp_segment<16>(k16, mask, a, e, q);
+            } else if (L <= 1024) {
+                unsigned k32[32];
+                warp_load_keys<32>(g, a, e, k32);
+                warp_segment<32>(k32, mask, a, e, q);
+            } else {
+                any_long = true;
+            }
+        }
     }
     // ---- longer segments: the whole block on one segment at a time
     if (__syncthreads_or(any_long)) {
         for (int s = 0; s < n_seg; ++s) {
             const int a = bounds[s], e = bounds[s + 1], q = quota[s], L = e - a;
             if (L <= 1024 || q <= 0 || q >= L) continue;
-            block_select(L, q, sh, round,
+            block_select<NT>(L, q, sh, round,
                          [&](int i) { return score_key(g[a + i]); },
                          [](int) { return true; },
                          [&](int i) { atomicOr(&mask[(a + i) >> 5], 1u << ((a + i) & 31)); });
@@ -787,7 +820,7 @@ __global__ void __launch_bounds__(kSelThreads, 4) k_select_compact(DevParams p)
     const int ns = max(0, min(p.n_sink, min(p.Tk, T)));
     const int nl = max(0, min(p.n_last, min(p.Tk - ns, T - ns)));
     int already = 0;
-    for (int i = tid; i < ns + nl; i += kSelThreads) {
+    for (int i = tid; i < ns + nl; i += NT) {
         const int t = i < ns ? i : T - nl + (i - ns);
         already += (atomicOr(&mask[t >> 5], 1u << (t & 31)) >> (t & 31)) & 1u;
     }
@@ -796,26 +829,26 @@ __global__ void __launch_bounds__(kSelThreads, 4) k_select_compact(DevParams p)
         auto key_at = [&](int t) { return score_key(g[t]); };
         auto unflagged = [&](int t) { return ((mask[t >> 5] >> (t & 31)) & 1u) == 0u; };
         auto raise = [&](int t) { atomicOr(&mask[t >> 5], 1u << (t & 31)); };
-        if (T <= kSelThreads * 16) {
+        if (T <= NT * 8) {
             // (winners are raised only after every thread has read its flags: the search ends with block-wide
             // counts before the first keep)
-            block_select(T, r_fill, sh, round, key_at, unflagged, raise);
+            block_select<NT>(T, r_fill, sh, round, key_at, unflagged, raise);
         } else {
             // Longer sequence: the r-th largest of the per-thread maxima is a lower bound of the r-th largest
             // key, so only tokens at or above it can win; they go to a short list.  Two walks over the scores
             // (float4 loads, four per thread in flight).
             const int T4 = (T + 3) & ~3;
             auto walk = [&](auto f) {
-                for (int base = 0; base < T4; base += kSelThreads * 16) {
+                for (int base = 0; base < T4; base += NT * 16) {
                     float4 v[4];
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const int t = base + (j * kSelThreads + tid) * 4;
+                        const int t = base + (j * NT + tid) * 4;
                         v[j] = t < T4 ? *reinterpret_cast<const float4 *>(g + t) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
                     }
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const int t = base + (j * kSelThreads + tid) * 4;
+                        const int t = base + (j * NT + tid) * 4;
                         if (t >= T4) continue;
                         const unsigned taken = mask[t >> 5] >> (t & 31); // (t is a multiple of 4: the four bits share a word)
                         const float x[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
@@ -832,15 +865,15 @@ __global__ void __launch_bounds__(kSelThreads, 4) k_select_compact(DevParams p)
             sh.tmax[tid] = tmax;
             __syncthreads();
             if (warp == 0) {
-                unsigned tv[kSelThreads / 32];
+                unsigned tv[NT / 32];
 #pragma unroll
-                for (int j = 0; j < kSelThreads / 32; ++j) tv[j] = sh.tmax[j * 32 + lane];
+                for (int j = 0; j < NT / 32; ++j) tv[j] = sh.tmax[j * 32 + lane];
                 unsigned M = 0;
                 for (int bit = 31; bit >= 0; --bit) {
                     const unsigned X = M | (1u << bit);
                     int c = 0;
 #pragma unroll
-                    for (int j = 0; j < kSelThreads / 32; ++j) c += tv[j] >= X;
+                    for (int j = 0; j < NT / 32; ++j) c += tv[j] >= X;
                     if (__reduce_add_sync(0xffffffffu, c) >= r_fill) M = X;
                 }
                 if (lane == 0) sh.bound = M;
@@ -886,14 +919,14 @@ __global__ void __launch_bounds__(kSelThreads, 4) k_select_compact(DevParams p)
                     }
                 }
             } else {
-                block_select_stream(T, r_fill, sh, round, key_at, unflagged, raise);
+                block_select_stream<NT>(T, r_fill, sh, round, key_at, unflagged, raise);
             }
         }
     }
     __syncthreads();
 
     // ---- ordered compaction of the kept positions: a thread takes a run of mask words
-    const int wpt = (n_words + kSelThreads - 1) / kSelThreads;
+    const int wpt = (n_words + NT - 1) / NT;
     const int w0 = tid * wpt, w1 = min(n_words, w0 + wpt);
     int n_kept = 0;
     for (int w = w0; w < w1; ++w) n_kept += __popc(mask[w]);
@@ -916,9 +949,9 @@ __global__ void __launch_bounds__(kSelThreads, 4) k_select_compact(DevParams p)
         float *credit = p.ema + (((size_t)un.l * p.Bmax + un.b) * p.H + un.h) * (size_t)p.T_cap;
         float *tmp = reinterpret_cast<float *>(p.cbuf + row); // the prefix sums are no longer needed
         __syncthreads();
-        for (int j = tid; j < p.Tk; j += kSelThreads) tmp[j] = credit[keep[j]];
+        for (int j = tid; j < p.Tk; j += NT) tmp[j] = credit[keep[j]];
         __syncthreads();
-        for (int j = tid; j < T; j += kSelThreads) credit[j] = j < p.Tk ? tmp[j] : 0.0f;
+        for (int j = tid; j < T; j += NT) credit[j] = j < p.Tk ? tmp[j] : 0.0f;
     }
 }
 
@@ -933,8 +966,13 @@ int launch_segsel(const DevParams &p, LaunchCtx &ctx)
 {
     const int units = p.L * p.B * p.H;
     const size_t smem_q = quota_smem(p.seg_cap, p.S).total, smem_s = sel_smem(p.T_cap, p.seg_cap).total;
-    static SmemGrant grant_q, grant_s;
-    if (!grant_dynamic_smem(k_segments_quotas, smem_q, grant_q) || !grant_dynamic_smem(k_select_compact, smem_s, grant_s))
+    // Long segments (no split, or a split length above a warp's reach) are searched by the whole block, one
+    // after the other, a barrier per key bit: four smaller blocks per SM hide that latency better; otherwise
+    // twice the warps per unit shorten the warp-per-segment phase.
+    const bool small_blocks = p.l_max == 0 || p.l_max > 1024;
+    static SmemGrant grant_q, grant_s256, grant_s512;
+    if (!grant_dynamic_smem(k_segments_quotas, smem_q, grant_q)) return AMS_ERR_CUDA;
+    if (small_blocks ? !grant_dynamic_smem(k_select_compact<256>, smem_s, grant_s256) : !grant_dynamic_smem(k_select_compact<512>, smem_s, grant_s512))
         return AMS_ERR_CUDA;
     const size_t smem_a = (size_t)(p.S + 1) * 8;
     if (ctx.launches <= 1) {
@@ -948,7 +986,9 @@ int launch_segsel(const DevParams &p, LaunchCtx &ctx)
     ctx.mark(kKernSegmentSelect);
     if (launch_after(k_segments_quotas, dim3((unsigned)units), dim3(32), smem_q, ctx.s, p) != cudaSuccess) return AMS_ERR_CUDA;
     ctx.mark(kKernQuota);
-    if (launch_after(k_select_compact, dim3((unsigned)units), dim3(kSelThreads), smem_s, ctx.s, p) != cudaSuccess) return AMS_ERR_CUDA;
+    const cudaError_t e3 = small_blocks ? launch_after(k_select_compact<256>, dim3((unsigned)units), dim3(256), smem_s, ctx.s, p)
+                                        : launch_after(k_select_compact<512>, dim3((unsigned)units), dim3(512), smem_s, ctx.s, p);
+    if (e3 != cudaSuccess) return AMS_ERR_CUDA;
     ctx.mark(kKernSelect);
     return AMS_OK;
 }

@@ -12,9 +12,7 @@ namespace sel {
 __device__ __forceinline__ float weight_of(float u, float eps)
 {
     // Eq. 1 numerator: max(u, 0) + eps; NaN counts as 0, +inf as FLT_MAX.
-    float v = __fadd_rn(fmaxf(u, 0.0f), eps);
-    if (!(v <= FLT_MAX)) v = FLT_MAX;
-    return v;
+    return fminf(__fadd_rn(fmaxf(u, 0.0f), eps), FLT_MAX); // (the sum is never NaN: fmaxf drops a NaN operand)
 }
 
 // 2^(kFixBits - (ilogb(mx) + 1)) as a double; mx > 0 (any fp32, subnormals included).
@@ -196,6 +194,20 @@ __device__ __forceinline__ float fixed_trunc(float x, int e)
     const int ef = max((int)((b >> 23) & 0xffu), 1); // subnormals share the scale of the smallest normal exponent
     const int n = e - (kFixBits - 23) - (ef - 127);
     return n <= 0 ? x : (n >= 24 ? 0.0f : __uint_as_float(b & (0xffffffffu << n)));
+}
+
+// The same truncation with two additions: below c = 2^(e - 13) a float is cut to a multiple of the image's
+// last bit 2^(e - 36) by adding c rounded down (sums in [c, 2c) have exactly that spacing) and taking c off
+// again (exact); from c upwards every float is such a multiple already.  c may be subnormal or zero for
+// tiny e: then every float is a multiple of the last bit and both branches return x.
+__device__ __forceinline__ float fixed_trunc_by_add(float x, float c)
+{
+    return x >= c ? x : __fsub_rn(__fadd_rd(x, c), c);
+}
+__device__ __forceinline__ float fixed_trunc_threshold(int e)
+{
+    const int k = e - (kFixBits - 23); // 2^k, any k in [-161, 115]
+    return k >= -126 ? __uint_as_float((unsigned)(k + 127) << 23) : (k >= -149 ? __uint_as_float(1u << (k + 149)) : 0.0f);
 }
 
 // 2^(kFixBits - e) as a double (e = fix_exponent of a positive fp32, so the result is a normal double).
