@@ -63,7 +63,19 @@ def _peaks():
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch from ncu captures summarised under
 # profiles/ (workload -> kernel slot -> bytes per launch).  A kernel or workload without a capture of the
 # current code reports null.
-NCU_TRAFFIC_BYTES: dict = {}
+NCU_TRAFFIC_BYTES: dict = {
+    # two-layer capture (profiles/tc_scorer_cfg4_2layers_ncu_full.md) x 40: the 80-layer launch holds 50 GB, too much to
+    # capture under full counters; units are independent and each is read once per pass, so traffic grows with the layers
+    "cfg4_llama70b_L80_T131072_k8192_w64": {"score_phase1": 40 * (540_693_760 + 5_705_216),
+                                            "score_phase2": 40 * (542_782_464 + 11_001_344)},
+    # captured at the timed size (profiles/tc_scorer_cfg1_32layers_ncu_full.md, profiles/gather_cfg1_cfg2_ncu_full.md)
+    "cfg1_llama8b_L32_T16384_k2048_w32": {"score_phase1": 1_089_466_880 + 13_675_520,
+                                          "score_phase2": 1_090_573_056 + 19_092_736,
+                                          "gather": 270_614_528 + 219_303_168},
+    # one-layer capture x 4 resident layers (profiles/keydiff_cfg3_1layer_ncu_full.md)
+    "cfg3_qwen3_8b_L36_B64_T32768_k2048_keydiff": {"score_phase1": 4 * (4_295_511_552 + 7_466_752),
+                                                   "score_phase2": 4 * (4_296_154_624 + 16_449_792)},
+}
 
 
 def config_dict(wl) -> dict:

@@ -19,6 +19,8 @@
 // which a block adds things up.  Selection order is (score key descending, position ascending), a strict
 // total order: the q-th element is found by fixing key bits from the top and, among keys equal to the
 // threshold, position bits.
+#include <type_traits>
+
 #include "ams_common.cuh"
 #include "ams_select.cuh"
 
@@ -42,12 +44,13 @@ __device__ __forceinline__ UnitId unit_of(const DevParams &p, int uid)
 
 // ------------------------------------------------------------------------------------------ k_mass_scan
 
-// Walks a row of `n4` floats (a multiple of 4) with float4 loads, four per thread in flight: f(t, v) gets the
-// position of the group's first element.  Thread and group order are the same in every call, so a thread
-// that wrote a group in one walk reads its own writes in the next.
+// Walks the first `n` floats of a row (allocated to a multiple of 4) with float4 loads, four per thread in
+// flight: f(t, v, full) gets the position of the group's first element and, as a compile-time flag, whether
+// the whole group lies inside the row (then no per-element bound is needed).
 template <typename F>
-__device__ __forceinline__ void walk4(const float *row, int n4, F f)
+__device__ __forceinline__ void walk4(const float *row, int n, F f)
 {
+    const int n4 = (n + 3) & ~3;
     const int tid = threadIdx.x;
     for (int base = 0; base < n4; base += kScanThreads * 16) {
         float4 v[4];
@@ -59,15 +62,17 @@ __device__ __forceinline__ void walk4(const float *row, int n4, F f)
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int t = base + (j * kScanThreads + tid) * 4;
-            if (t < n4) f(t, v[j]);
+            if (t + 3 < n) f(t, v[j], std::true_type{});
+            else if (t < n) f(t, v[j], std::false_type{});
         }
     }
 }
 
 // The same over two rows at once (usage and credit).
 template <typename F>
-__device__ __forceinline__ void walk4x2(const float *row_a, const float *row_b, int n4, F f)
+__device__ __forceinline__ void walk4x2(const float *row_a, const float *row_b, int n, F f)
 {
+    const int n4 = (n + 3) & ~3;
     const int tid = threadIdx.x;
     for (int base = 0; base < n4; base += kScanThreads * 16) {
         float4 va[4], vb[4];
@@ -80,7 +85,8 @@ __device__ __forceinline__ void walk4x2(const float *row_a, const float *row_b, 
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int t = base + (j * kScanThreads + tid) * 4;
-            if (t < n4) f(t, va[j], vb[j]);
+            if (t + 3 < n) f(t, va[j], vb[j], std::true_type{});
+            else if (t < n) f(t, va[j], vb[j], std::false_type{});
         }
     }
 }
@@ -128,13 +134,12 @@ __global__ void __launch_bounds__(kScanThreads) k_mass_scan(DevParams p)
 
     // Rows are allocated to the capacity (a multiple of 16), so whole float4 groups may be read past the
     // sequence's end; what lies there is masked by position.
-    const int T4 = (T + 3) & ~3;
     // ---- largest Eq. 1 weight -> exponent of the fixed-point images
     float wmax = 0.0f;
-    walk4(u, T4, [&](int t, float4 v) {
+    walk4(u, T, [&](int t, float4 v, auto full) {
         const float w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-        for (int i = 0; i < 4; ++i) if (t + i < T) wmax = fmaxf(wmax, weight_of(w[i], p.eps));
+        for (int i = 0; i < 4; ++i) if (decltype(full)::value || t + i < T) wmax = fmaxf(wmax, weight_of(w[i], p.eps));
     });
     wmax = block_max_f32(wmax, scratch);
     const int ew = fix_exponent(wmax);
@@ -142,11 +147,11 @@ __global__ void __launch_bounds__(kScanThreads) k_mass_scan(DevParams p)
     const double scale_w = fix_scale_of(ew);
     const float cut_w = fixed_trunc_threshold(ew); // weights below it lose their bits under the image's last one
     double sa = 0.0;
-    walk4(u, T4, [&](int t, float4 v) {
+    walk4(u, T, [&](int t, float4 v, auto full) {
         const float w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-            if (t + i < T) sa = __dadd_rn(sa, __dmul_rn((double)fixed_trunc_by_add(weight_of(w[i], p.eps), cut_w), scale_w));
+            if (decltype(full)::value || t + i < T) sa = __dadd_rn(sa, __dmul_rn((double)fixed_trunc_by_add(weight_of(w[i], p.eps), cut_w), scale_w));
     });
     const double SA = block_sum_exact_f64(sa, scratch);
     const double inv_sa = __ddiv_rn(1.0, SA);          // normalisations multiply by the rounded reciprocal
@@ -161,19 +166,19 @@ __global__ void __launch_bounds__(kScanThreads) k_mass_scan(DevParams p)
     if (ema_on) {
         const float oml = __fsub_rn(1.0f, p.lambda);
         float cmax = 0.0f;
-        walk4x2(u, credit, T4, [&](int t, float4 v, float4 cv) {
+        walk4x2(u, credit, T, [&](int t, float4 v, float4 cv, auto full) {
             const float w[4] = {v.x, v.y, v.z, v.w};
             float c[4] = {cv.x, cv.y, cv.z, cv.w};
             float m[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 m[i] = __double2float_rn(__dmul_rn((double)fixed_trunc_by_add(weight_of(w[i], p.eps), cut_w), inv_sa_w));
-                if (t + i < T) {
+                if (decltype(full)::value || t + i < T) {
                     c[i] = __fadd_rn(__fmul_rn(p.lambda, c[i]), __fmul_rn(oml, m[i]));
                     cmax = fmaxf(cmax, c[i]);
                 }
             }
-            if (t + 3 < T) {
+            if (decltype(full)::value) {
                 *reinterpret_cast<float4 *>(credit + t) = make_float4(c[0], c[1], c[2], c[3]);
                 if (mass_dbg) *reinterpret_cast<float4 *>(mass_dbg + t) = make_float4(m[0], m[1], m[2], m[3]);
             } else {
@@ -189,11 +194,11 @@ __global__ void __launch_bounds__(kScanThreads) k_mass_scan(DevParams p)
             ec = fix_exponent(cmax);
             scale_c = fix_scale_of(ec);
             cut_c = fixed_trunc_threshold(ec);
-            walk4(credit, T4, [&](int t, float4 cv) {
+            walk4(credit, T, [&](int t, float4 cv, auto full) {
                 const float c[4] = {cv.x, cv.y, cv.z, cv.w};
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
-                    if (t + i < T) scsum = __dadd_rn(scsum, __dmul_rn((double)fixed_trunc_by_add(c[i], cut_c), scale_c));
+                    if (decltype(full)::value || t + i < T) scsum = __dadd_rn(scsum, __dmul_rn((double)fixed_trunc_by_add(c[i], cut_c), scale_c));
             });
         }
         const double SC = block_sum_exact_f64(scsum, scratch);

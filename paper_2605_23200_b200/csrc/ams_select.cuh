@@ -164,7 +164,7 @@ __device__ void radix_select(const float *g, int a, int b, int k, int *hist, int
     *ties = n_ties;
 }
 
-// ---- the same fixed-point images without 64-bit conversions -------------------------------
+// ---- fixed-point images through fp32 / fp64 arithmetic (the three-kernel form) -----------------
 // Exponent e = ilogb(mx) + 1 of the largest weight mx > 0 (any fp32, subnormals included).
 __device__ __forceinline__ int fix_exponent(float mx)
 {
@@ -172,31 +172,12 @@ __device__ __forceinline__ int fix_exponent(float mx)
     return (int)((bits >> 52) & 0x7ff) - 1023 + 1;
 }
 
-// floor(x * 2^(kFixBits - e)) for 0 <= x < 2^e, from the bits of x: x = m * 2^(E - 23) with a
-// 24-bit integer m, so the image is m shifted by E + 13 - e (at most 12 to the left).
-__device__ __forceinline__ u64 to_fixed_bits(float x, int e)
-{
-    const unsigned b = __float_as_uint(x);
-    const int ef = (int)((b >> 23) & 0xffu);
-    const u64 m = ef ? ((b & 0x7fffffu) | 0x800000u) : (b & 0x7fffffu);
-    const int sh = (ef ? ef - 127 : -126) + (kFixBits - 23) - e;
-    return sh >= 0 ? (m << sh) : (sh > -24 ? (m >> (-sh)) : 0ull);
-}
-
 // The fixed-point image A = floor(x * 2^(kFixBits - e)) (0 <= x < 2^e) equals trunc(x) * 2^(kFixBits - e), where
 // trunc(x) is x with the mantissa bits below the image's last bit cleared: x = m * 2^(E - 23), and the image
 // drops the lowest n = e - 13 - E bits of m when that is positive (all 24 of them from n = 24 on).  So the
 // image is available as a double with one conversion and one exact multiplication by a power of two, and
 // sums of images (integers below 2^53) can be added in fp64 in any order.
-__device__ __forceinline__ float fixed_trunc(float x, int e)
-{
-    const unsigned b = __float_as_uint(x);
-    const int ef = max((int)((b >> 23) & 0xffu), 1); // subnormals share the scale of the smallest normal exponent
-    const int n = e - (kFixBits - 23) - (ef - 127);
-    return n <= 0 ? x : (n >= 24 ? 0.0f : __uint_as_float(b & (0xffffffffu << n)));
-}
-
-// The same truncation with two additions: below c = 2^(e - 13) a float is cut to a multiple of the image's
+// The truncation takes two additions: below c = 2^(e - 13) a float is cut to a multiple of the image's
 // last bit 2^(e - 36) by adding c rounded down (sums in [c, 2c) have exactly that spacing) and taking c off
 // again (exact); from c upwards every float is such a multiple already.  c may be subnormal or zero for
 // tiny e: then every float is a multiple of the last bit and both branches return x.
@@ -214,12 +195,6 @@ __device__ __forceinline__ float fixed_trunc_threshold(int e)
 __device__ __forceinline__ double fix_scale_of(int e)
 {
     return __longlong_as_double((long long)(1023 + kFixBits - e) << 52);
-}
-
-// (double)a for an integer a < 2^52, exact.
-__device__ __forceinline__ double u52_to_double(u64 a)
-{
-    return __dsub_rn(__longlong_as_double((long long)(0x4330000000000000ull | a)), 4503599627370496.0);
 }
 
 // floor(y) for 0 <= y < 2^51 as an integer: y + 2^52 rounded down lands on the integer grid.
