@@ -68,6 +68,13 @@ EXT_CASES = [
     # ragged with skipped sequences, and a budget that is not a multiple of the page size
     ("lognormal", dict(n_layers=4, batch=9, seq_len_min=500, seq_len_max=2600, budget=1203, n_last=5)),
     ("ties", dict(n_layers=5, batch=4, seq_len_min=4000, seq_len_max=9000, budget=2048, ema_beta=1.0, n_segments=12)),
+    # backfill on a long sequence whose candidates all tie (the short candidate list overflows: every round re-reads the scores)
+    ("constant", dict(seq_len_min=20000, seq_len_max=20000, budget=3000, batch=1, n_layers=1)),
+    ("ties", dict(seq_len_min=21003, seq_len_max=21003, budget=2500, batch=1, n_layers=1, n_sink=40, n_last=300)),
+    # NaN, infinities and signed zeros on a long sequence (keys of zero in the candidate search), long unsplit segments
+    ("signed_nan", dict(seq_len_min=19001, seq_len_max=19001, budget=2048, batch=2, n_layers=1, ema_beta=1.0, l_max=0, n_segments=6)),
+    # many more must-keep positions than a block has threads (backfill count above the per-thread maxima's reach)
+    ("lognormal", dict(seq_len_min=12000, seq_len_max=12000, budget=4000, batch=1, n_layers=1, n_sink=900, n_last=1200, l_max=1024)),
 ]
 
 
