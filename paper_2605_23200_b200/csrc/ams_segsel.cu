@@ -541,15 +541,18 @@ struct SelShared {
 // Sum of one count per thread over the block with one barrier per call: counts of consecutive calls land in
 // alternating tables, so a table is rewritten only after every thread has passed the barrier that follows
 // its last read.
-template <int NT>
+template <int NT, int GT = NT>
 __device__ __forceinline__ int block_count(int c, int round, SelShared &sh)
 {
-    const int lane = threadIdx.x & 31;
+    // GT = NT: the whole block counts together; GT < NT: the block's teams of GT threads count on their own, each
+    // behind its own named barrier (teams never share a warp's table entry)
+    const int lane = threadIdx.x & 31, team = threadIdx.x / GT;
     c = __reduce_add_sync(0xffffffffu, c);
     int *mine = sh.wc[round & 1];
     if (lane == 0) mine[threadIdx.x >> 5] = c;
-    __syncthreads();
-    const int v = lane < NT / 32 ? mine[lane] : 0;
+    if (GT == NT) __syncthreads();
+    else asm volatile("bar.sync %0, %1;" ::"r"(1 + team), "n"(GT) : "memory");
+    const int v = lane < GT / 32 ? mine[team * (GT / 32) + lane] : 0;
     return __reduce_add_sync(0xffffffffu, v);
 }
 
@@ -623,15 +626,15 @@ __device__ __forceinline__ void warp_segment(const unsigned (&k)[KPL], unsigned 
 // j * NT + tid (numbers ascend with position).  key_of(i) gives the score key, ok(i) whether the item
 // takes part; keep(i) is called for every winner.  First the key bits, then (if more than q items lie at or
 // above the q-th key) the item numbers of the tied items, smaller first.
-template <int NT, int KPT, typename KeyOf, typename Ok, typename Keep>
+template <int NT, int GT, int KPT, typename KeyOf, typename Ok, typename Keep>
 __device__ __forceinline__ void block_select_reg(int n, int q, SelShared &sh, int &round, KeyOf key_of, Ok ok, Keep keep)
 {
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x % GT; // position inside the counting group
     unsigned k[KPT];
     unsigned elig = 0;
 #pragma unroll
     for (int j = 0; j < KPT; ++j) {
-        const int i = j * NT + tid;
+        const int i = j * GT + tid;
         k[j] = 0u;
         if (i < n && ok(i)) { elig |= 1u << j; k[j] = key_of(i); }
     }
@@ -642,7 +645,7 @@ __device__ __forceinline__ void block_select_reg(int n, int q, SelShared &sh, in
         int c = 0;
 #pragma unroll
         for (int j = 0; j < KPT; ++j) c += k[j] >= X;
-        const int tot = block_count<NT>(c, round++, sh);
+        const int tot = block_count<NT, GT>(c, round++, sh);
         if (tot >= q) {
             P = X;
             if (tot == q) { exact = true; break; }
@@ -655,12 +658,12 @@ __device__ __forceinline__ void block_select_reg(int n, int q, SelShared &sh, in
     if (!exact) {
         // ties at the threshold: the first (q - #above) of them by item number.  Search the item-number image
         // n - i (larger = earlier), unique per item, so the count ends exactly.
-        const int above = block_count<NT>(__popc(win), round++, sh);
+        const int above = block_count<NT, GT>(__popc(win), round++, sh);
         const int take = q - above;
         unsigned tie = 0;
 #pragma unroll
         for (int j = 0; j < KPT; ++j) {
-            const int i = j * NT + tid;
+            const int i = j * GT + tid;
             const bool is_tie = ((elig >> j) & 1u) && k[j] == P;
             if (is_tie) tie |= 1u << j;
             k[j] = is_tie ? (unsigned)(n - i) : 0u;
@@ -671,7 +674,7 @@ __device__ __forceinline__ void block_select_reg(int n, int q, SelShared &sh, in
             int c = 0;
 #pragma unroll
             for (int j = 0; j < KPT; ++j) c += k[j] >= X;
-            const int tot = block_count<NT>(c, round++, sh);
+            const int tot = block_count<NT, GT>(c, round++, sh);
             if (tot >= take) {
                 P2 = X;
                 if (tot == take) break;
@@ -683,7 +686,7 @@ __device__ __forceinline__ void block_select_reg(int n, int q, SelShared &sh, in
     }
 #pragma unroll
     for (int j = 0; j < KPT; ++j)
-        if ((win >> j) & 1u) keep(j * NT + tid);
+        if ((win >> j) & 1u) keep(j * GT + tid);
 }
 
 // The same selection for sets too large for registers: every round walks the items again (scores from L2).
@@ -729,10 +732,10 @@ __device__ void block_select_stream(int n, int q, SelShared &sh, int &round, Key
 template <int NT, typename KeyOf, typename Ok, typename Keep>
 __device__ __forceinline__ void block_select(int n, int q, SelShared &sh, int &round, KeyOf key_of, Ok ok, Keep keep)
 {
-    if (n <= NT * 4) block_select_reg<NT, 4>(n, q, sh, round, key_of, ok, keep);
-    else if (n <= NT * 8) block_select_reg<NT, 8>(n, q, sh, round, key_of, ok, keep);
-    else if (n <= NT * 16) block_select_reg<NT, 16>(n, q, sh, round, key_of, ok, keep);
-    else if (NT <= 256 && n <= NT * 32) block_select_reg<NT, NT <= 256 ? 32 : 16>(n, q, sh, round, key_of, ok, keep);
+    if (n <= NT * 4) block_select_reg<NT, NT, 4>(n, q, sh, round, key_of, ok, keep);
+    else if (n <= NT * 8) block_select_reg<NT, NT, 8>(n, q, sh, round, key_of, ok, keep);
+    else if (n <= NT * 16) block_select_reg<NT, NT, 16>(n, q, sh, round, key_of, ok, keep);
+    else if (NT <= 256 && n <= NT * 32) block_select_reg<NT, NT, NT <= 256 ? 32 : 16>(n, q, sh, round, key_of, ok, keep);
     else block_select_stream<NT>(n, q, sh, round, key_of, ok, keep);
 }
 
@@ -807,15 +810,32 @@ __global__ void __launch_bounds__(NT, 1024 / NT) k_select_compact(DevParams p)
             }
         }
     }
-    // ---- longer segments: the whole block on one segment at a time
+    // ---- longer segments: teams of four warps take those of up to 4096 tokens in turn, each team behind its own
+    //      barrier (a count per key bit costs a team a fraction of a block-wide barrier, and the teams search
+    //      different segments at the same time); the whole block then takes what is longer still
     if (__syncthreads_or(any_long)) {
-        for (int s = 0; s < n_seg; ++s) {
-            const int a = bounds[s], e = bounds[s + 1], q = quota[s], L = e - a;
-            if (L <= 1024 || q <= 0 || q >= L) continue;
+        constexpr int GT = 128, kTeamMax = GT * 32;
+        const int team = tid / GT;
+        int k = 0;
+        for (int sg = 0; sg < n_seg; ++sg) {
+            const int a = bounds[sg], e = bounds[sg + 1], q = quota[sg], L = e - a;
+            if (L <= 1024 || L > kTeamMax || q <= 0 || q >= L) continue;
+            if (k++ % (NT / GT) != team) continue;
+            auto key_of = [&](int i) { return score_key(g[a + i]); };
+            auto all = [](int) { return true; };
+            auto keepit = [&](int i) { atomicOr(&mask[(a + i) >> 5], 1u << ((a + i) & 31)); };
+            if (L <= GT * 16) block_select_reg<NT, GT, 16>(L, q, sh, round, key_of, all, keepit);
+            else block_select_reg<NT, GT, 32>(L, q, sh, round, key_of, all, keepit);
+        }
+        __syncthreads();
+        round = 0; // the teams counted different numbers of rounds: everybody starts the block-wide counts on the same table
+        for (int sg = 0; sg < n_seg; ++sg) {
+            const int a = bounds[sg], e = bounds[sg + 1], q = quota[sg], L = e - a;
+            if (L <= kTeamMax || q <= 0 || q >= L) continue;
             block_select<NT>(L, q, sh, round,
-                         [&](int i) { return score_key(g[a + i]); },
-                         [](int) { return true; },
-                         [&](int i) { atomicOr(&mask[(a + i) >> 5], 1u << ((a + i) & 31)); });
+                             [&](int i) { return score_key(g[a + i]); },
+                             [](int) { return true; },
+                             [&](int i) { atomicOr(&mask[(a + i) >> 5], 1u << ((a + i) & 31)); });
         }
         __syncthreads();
     }
