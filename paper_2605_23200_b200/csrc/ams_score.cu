@@ -275,6 +275,26 @@ __global__ void __launch_bounds__(256) k_tova_usage_from_logits(DevParams p)
 
 constexpr int kKdThreads = 256; // 16 token rows x 16 lanes of 16 bytes
 
+// Packed fp32 pairs (two floats in a 64-bit register) and their fused multiply-add.
+__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi)
+{
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ unsigned long long fma_f32x2(unsigned long long a, unsigned long long b, unsigned long long c)
+{
+    unsigned long long r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ float sum_f32x2(unsigned long long a)
+{
+    float lo, hi;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(a));
+    return lo + hi;
+}
+
 __global__ void __launch_bounds__(kKdThreads) k_keydiff_sum(DevParams p)
 {
     __shared__ float red[16][kHeadDim];
@@ -340,9 +360,9 @@ __global__ void __launch_bounds__(kKdThreads) k_keydiff_score(DevParams p)
     const int lane = threadIdx.x & 15, r = threadIdx.x >> 4;
     const int *table = p.block_table + (size_t)b * p.bt_stride;
     const float *fin = p.fin + (size_t)uid * (p.rows_pad + 8);
-    float mu[8];
+    unsigned long long mu2[4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) mu[i] = fin[lane * 8 + i];
+    for (int i = 0; i < 4; ++i) mu2[i] = pack_f32x2(fin[lane * 8 + 2 * i], fin[lane * 8 + 2 * i + 1]);
     const float mu_norm = fin[kHeadDim];
     float *g_out = p.scores + (size_t)uid * p.T_cap;
     // four tokens per thread and round: their loads are issued together, so that enough bytes are in flight
@@ -360,12 +380,17 @@ __global__ void __launch_bounds__(kKdThreads) k_keydiff_score(DevParams p)
         float a[2 * kU];
 #pragma unroll
         for (int u = 0; u < kU; ++u) {
-            const float k[8] = {bf16_lo(v[u].x), bf16_hi(v[u].x), bf16_lo(v[u].y), bf16_hi(v[u].y),
-                                bf16_lo(v[u].z), bf16_hi(v[u].z), bf16_lo(v[u].w), bf16_hi(v[u].w)};
-            float dot = 0.0f, k2 = 0.0f;
+            // two dimensions per instruction: a bf16 pair widens to a packed fp32 pair (low half shifted up, high half
+            // masked), and both running sums take packed multiply-adds
+            const unsigned w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+            unsigned long long dot2 = 0ull, sq2 = 0ull; // (0.0f, 0.0f)
 #pragma unroll
-            for (int i = 0; i < 8; ++i) { dot = fmaf(k[i], mu[i], dot); k2 = fmaf(k[i], k[i], k2); }
-            a[2 * u] = dot; a[2 * u + 1] = k2;
+            for (int i = 0; i < 4; ++i) {
+                const unsigned long long k2 = pack_f32x2(bf16_lo(w[i]), bf16_hi(w[i]));
+                dot2 = fma_f32x2(k2, mu2[i], dot2);
+                sq2 = fma_f32x2(k2, k2, sq2);
+            }
+            a[2 * u] = sum_f32x2(dot2); a[2 * u + 1] = sum_f32x2(sq2);
         }
         // sums over the 16 lanes of a token row, all eight values at once: at each step a lane hands half of
         // its values to its partner and keeps the other half (9 shuffles instead of 32)
