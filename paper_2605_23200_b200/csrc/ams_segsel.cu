@@ -450,6 +450,7 @@ __global__ void __launch_bounds__(32) k_segments_quotas(DevParams p)
         n_merged = nm - 1;
         n_seg = off;
     }
+    __syncwarp(); // lane 0's tables are read by every lane below
     n_merged = __shfl_sync(0xffffffffu, n_merged, 0);
     n_seg = __shfl_sync(0xffffffffu, n_seg, 0);
     if (n_seg > sc) { // cannot happen with the capacity formula of the header; reported all the same
