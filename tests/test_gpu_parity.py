@@ -311,3 +311,39 @@ def test_event_captured_in_a_cuda_graph_replays_identically():
             assert torch.equal(a.view(torch.int16) if a.dtype == torch.bfloat16 else a,
                                b.view(torch.int16) if b.dtype == torch.bfloat16 else b)
         restore()
+
+
+def test_stored_small_case_two_events():
+    """The library against tests/golden/select_unit_small.json (written by the oracle alone): two consecutive events
+    on caller-supplied scores with the credit carried through the compaction."""
+    import importlib.util
+    import json
+    import os
+    here = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+    spec = importlib.util.spec_from_file_location("make_golden", os.path.join(here, "make_golden.py"))
+    mg = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mg)
+    gold = json.load(open(os.path.join(here, "select_unit_small.json")))
+    prm = gold["params"]
+    wl = inputs.CONFIGS[0].scaled(n_layers=1, batch=1, n_q_heads=1, n_kv_heads=1, seq_len_min=gold["T"], seq_len_max=gold["T"],
+                                  budget=gold["Tk"], append_per_step=gold["append"], steps=2, resident_layers=0, **prm)
+    cache = inputs.make_cache(wl, DEV)
+    comp = binding.AmsCompressor(binding.config_for(wl), DEV)
+    for event, want in enumerate(gold["events"]):
+        n = want["n_tokens"]
+        assert int(cache.seq_lens[0]) == n
+        ext = np.zeros((1, 1, 1, wl.max_seq_len), np.float32)
+        ext[0, 0, 0, :n] = mg.scores(event, n)
+        dst = inputs.alloc_dst_pages(cache)
+        dbg = gpu_event(comp, cache, dst, inputs.SCORER_EXTERNAL, torch.from_numpy(ext).to(DEV))
+        ns = int(dbg.n_segments[0, 0, 0])
+        assert ns == want["n_seg"]
+        assert dbg.seg_bounds[0, 0, 0, : ns + 1].cpu().tolist() == want["bounds"]
+        assert dbg.quotas[0, 0, 0, :ns].cpu().tolist() == want["quotas"]
+        assert dbg.keep_idx[0, 0, 0].cpu().tolist() == want["keep_idx"]
+        assert dbg.mass[0, 0, 0, :8].cpu().numpy().view(np.uint32).tolist() == want["mass_bits_first8"]
+        assert comp.ema_state[0, 0, 0, :8].cpu().numpy().view(np.uint32).tolist() == want["credit_bits_first8"]
+        assert abs(float(comp.ema_state[0, 0, 0].double().sum()) - want["credit_sum_f64"]) < 1e-12
+        inputs.after_compress(cache, dst)
+        if event == 0:
+            inputs.append_tokens(cache, wl.append_per_step)

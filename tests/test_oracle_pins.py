@@ -723,3 +723,30 @@ def test_retained_iou_closed_forms():
     assert oracle.retained_iou(keep, Tk, Tk) == np.float32(4) / np.float32(12)
     assert oracle.retained_iou(keep, 0, Tk) == np.float32(0.0)                           # no previous event
     assert oracle.retained_iou(keep, 5, Tk) == np.float32(3) / np.float32(10)            # a smaller previous budget
+
+
+# ----------------------------------------------------------------------------- stored results
+
+def test_oracle_reproduces_the_stored_small_case():
+    """tests/golden/select_unit_small.json was written by tests/golden/make_golden.py from the oracle alone; an
+    accidental change to the oracle's arithmetic or tie rules shows up here."""
+    import importlib.util
+    import json
+    import os
+    here = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+    spec = importlib.util.spec_from_file_location("make_golden", os.path.join(here, "make_golden.py"))
+    mg = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mg)
+    gold = json.load(open(os.path.join(here, "select_unit_small.json")))
+    prm = Params(**gold["params"])
+    credit = np.zeros(gold["T"], np.float32)
+    for event, want in enumerate(gold["events"]):
+        n = want["n_tokens"]
+        u = mg.scores(event, n)
+        r = oracle.select_unit(u, u, credit[:n], gold["Tk"], prm)
+        assert r.bounds.tolist() == want["bounds"] and r.quotas.tolist() == want["quotas"]
+        assert r.keep_idx.tolist() == want["keep_idx"] and r.n_backfill == want["n_backfill"]
+        assert [int(v) for v in r.mass[:8].view(np.uint32)] == want["mass_bits_first8"]
+        assert [int(v) for v in r.credit[:8].view(np.uint32)] == want["credit_bits_first8"]
+        credit = np.zeros(gold["Tk"] + gold["append"], np.float32)
+        credit[: gold["Tk"]] = r.credit[: gold["Tk"]]
