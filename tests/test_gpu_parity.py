@@ -73,6 +73,12 @@ EXT_CASES = [
     ("ties", dict(seq_len_min=21003, seq_len_max=21003, budget=2500, batch=1, n_layers=1, n_sink=40, n_last=300)),
     # NaN, infinities and signed zeros on a long sequence (keys of zero in the candidate search), long unsplit segments
     ("signed_nan", dict(seq_len_min=19001, seq_len_max=19001, budget=2048, batch=2, n_layers=1, ema_beta=1.0, l_max=0, n_segments=6)),
+    # the smallest geometry (one page) and a few tokens more than the budget
+    ("lognormal", dict(seq_len_min=16, seq_len_max=16, budget=5, batch=2, n_layers=1, n_segments=3, l_min=2, l_max=8, n_sink=1, n_last=2)),
+    ("ties", dict(seq_len_min=41, seq_len_max=41, budget=40, batch=1, n_layers=2, n_segments=10)),
+    # thousands of tiny segments on a long sequence (segment tables near their capacity)
+    ("ties", dict(seq_len_min=30000, seq_len_max=30000, budget=9000, batch=1, n_layers=1, n_kv_heads=2, n_q_heads=8, l_min=1, l_max=17,
+                  n_segments=64, q_min=2)),
     # many more must-keep positions than a block has threads (backfill count above the per-thread maxima's reach)
     ("lognormal", dict(seq_len_min=12000, seq_len_max=12000, budget=4000, batch=1, n_layers=1, n_sink=900, n_last=1200, l_max=1024)),
 ]
