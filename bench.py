@@ -74,7 +74,7 @@ NCU_TRAFFIC_BYTES: dict = {
                                           "gather": 270_614_528 + 219_303_168},
     # one-layer capture x 4 resident layers (profiles/keydiff_cfg3_1layer_ncu_full.md)
     "cfg3_qwen3_8b_L36_B64_T32768_k2048_keydiff": {"score_phase1": 4 * (4_295_511_552 + 7_466_752),
-                                                   "score_phase2": 4 * (4_296_154_624 + 16_449_792)},
+                                                   "score_phase2": 4 * (4_296_070_144 + 16_274_688)},
 }
 
 
