@@ -82,6 +82,7 @@ def lib():
         _lib.orc_select.restype = ctypes.c_int32
         _lib.orc_score_tova.restype = ctypes.c_int
         _lib.orc_score_keydiff.restype = ctypes.c_int
+        _lib.orc_score_expected.restype = ctypes.c_int
     return _lib
 
 
@@ -124,6 +125,28 @@ def score_keydiff(k_pages, layer, h, table_row, T):
                                  _p(out, ctypes.c_float))
     if rc != 0:
         raise ValueError(f"orc_score_keydiff failed: {rc}")
+    return out
+
+
+def score_expected(k_pages, v_pages, layer, h, table_row, T, mean, cov, eps):
+    """Expected-attention score of one (layer, sequence, KV head): Gaussian closed form of the
+    expected attention weight per query head of the group, softmax over the tokens, group
+    mean, (+ eps) times the value norm (the scorer of the paper's "AMS-Expected" rows; the
+    formula is a reading, see ams_oracle.c).  mean: float32 [G][D]; cov: uint16 (bf16) [G][D][D]."""
+    L, P, page, H, D = k_pages.shape
+    table_row = _i32(table_row)
+    mean = _f32(mean)
+    cov = np.ascontiguousarray(cov, dtype=np.uint16)
+    G = mean.shape[0]
+    assert mean.shape == (G, D) and cov.shape == (G, D, D)
+    out = np.empty(T, dtype=np.float32)
+    rc = lib().orc_score_expected(_p(k_pages, ctypes.c_uint16), _p(v_pages, ctypes.c_uint16), ctypes.c_int64(P),
+                                  ctypes.c_int32(page), ctypes.c_int32(H), ctypes.c_int32(D), ctypes.c_int32(layer),
+                                  ctypes.c_int32(h), _p(table_row, ctypes.c_int32), ctypes.c_int32(T),
+                                  _p(mean, ctypes.c_float), _p(cov, ctypes.c_uint16), ctypes.c_int32(G),
+                                  ctypes.c_float(eps), _p(out, ctypes.c_float))
+    if rc != 0:
+        raise ValueError(f"orc_score_expected failed: {rc}")
     return out
 
 
@@ -288,12 +311,13 @@ def retained_iou(keep_idx, prev_kept, budget):
 
 # --------------------------------------------------------------------------- whole event
 
-SCORER_TOVA, SCORER_KEYDIFF, SCORER_EXTERNAL = 0, 1, 2
+SCORER_TOVA, SCORER_KEYDIFF, SCORER_EXTERNAL, SCORER_EXPECTED = 0, 1, 2, 3
 
 
 def compress(k_pages, v_pages, block_table, seq_lens, obs_queries, credit, budget, prm: Params,
              scorer_id, dst_pages, *, n_q_heads=None, causal=True, ext_scores=None, units=None,
-             do_gather=True, threads=1, pool_kernel=1, decoupled=False, ext_usage=None):
+             do_gather=True, threads=1, pool_kernel=1, decoupled=False, ext_usage=None, q_mean=None, q_cov=None,
+             score_eps=1e-2):
     """One compression event over every layer, sequence and KV head.
 
     k_pages / v_pages: uint16 [L][P][page][H][D] (modified: kept rows are written into
@@ -325,6 +349,12 @@ def compress(k_pages, v_pages, block_table, seq_lens, obs_queries, credit, budge
         elif scorer_id == SCORER_KEYDIFF:
             s = score_keydiff(k_pages, l, h, block_table[b], T)
             if decoupled:
+                W = obs_queries.shape[3]
+                u = score_tova(k_pages, l, h, block_table[b], T, obs_queries[l, b, h * G:(h + 1) * G], G, W, causal)
+        elif scorer_id == SCORER_EXPECTED:
+            s = score_expected(k_pages, v_pages, l, h, block_table[b], T, q_mean[l, b, h * G:(h + 1) * G],
+                               q_cov[l, b, h * G:(h + 1) * G], score_eps)
+            if decoupled and obs_queries is not None:
                 W = obs_queries.shape[3]
                 u = score_tova(k_pages, l, h, block_table[b], T, obs_queries[l, b, h * G:(h + 1) * G], G, W, causal)
         else:

@@ -25,7 +25,9 @@
  * the budget with their bounds; one segment => library top-k; beta = 1 => EMA
  * off; lambda = 0 => credit equals mass; gather equals dense indexing; TOVA
  * with one query row => library softmax; KeyDiff => library cosine similarity;
- * usage smoothing => library zero-padded average pooling and a hand-computed case.
+ * usage smoothing => library zero-padded average pooling and a hand-computed case;
+ * expected-attention logits => Monte-Carlo mean of exp(q.k/sqrt(D)) over sampled Gaussian
+ * queries, zero covariance => the one-query TOVA softmax, isotropic covariance => closed form.
  * EMA weights (beta on the current mass, 1 - beta on the normalised credit) and
  * the must-keep order (suffix gives way before the sinks) against exact rationals
  * and hand-worked cases; quota rounding (halves up) and the visiting order of the
@@ -34,7 +36,9 @@
  * Parity unpinned (invariants and hand-made examples of this reading only, the
  * paper fixes neither): merge direction and the order of merge vs split; the
  * choice of "roughly equal" split sizes; the padding value of the causal
- * observation window when W > 1.
+ * observation window when W > 1; for the expected-attention score, the order
+ * softmax -> group mean -> (+ eps) -> value norm (the paper prints no formula; the
+ * Gaussian closed form itself is pinned to its definition).
  */
 #include <float.h>
 #include <math.h>
@@ -174,6 +178,67 @@ int orc_score_keydiff(const uint16_t *pages, int64_t num_pages, int32_t page_siz
         g_out[t] = (float)(-dot / den);
     }
     free(mu);
+    return 0;
+}
+
+static const uint16_t *v_row(const orc_pool *P, int layer, const int32_t *table_row, int t, int h)
+{
+    return P->pages + row_offset(P, layer, table_row[t / P->page_size], t % P->page_size, h);
+}
+
+/* Expected-attention score (the scorer behind the paper's "AMS-Expected" rows; the
+ * paper names it, its regularisation coefficient epsilon = 1e-2 and the work it comes
+ * from, but prints no formula: what follows is a READING, the closed form that the
+ * cited work's idea gives when the future queries of a head are modelled as Gaussian).
+ * For a query q ~ N(mu, Sigma) the expected unnormalised attention weight of key k is
+ * the Gaussian moment-generating function
+ *     E[exp(q.k / sqrt(D))] = exp(mu.k / sqrt(D) + k^T Sigma k / (2 D)).
+ * Per query head r of the KV head's GQA group: logit l_{r,t} = mu_r.k_t / sqrt(D) +
+ * k_t^T Sigma_r k_t / (2 D), softmax over the T cached tokens, mean over the G heads of
+ * the group, then (a_t + eps) * |v_t|_2 (the value norm weighs what a token would
+ * contribute).  The query statistics are inputs (they come from the model's hidden
+ * states, outside this step): mean fp32 [G][D], cov bf16 [G][D][D] (need not be
+ * symmetric: only its symmetric part matters to the quadratic form). */
+int orc_score_expected(const uint16_t *k_pages, const uint16_t *v_pages, int64_t num_pages, int32_t page_size,
+                       int32_t n_kv_heads, int32_t head_dim, int32_t layer, int32_t h, const int32_t *table_row,
+                       int32_t T, const float *mean, const uint16_t *cov, int32_t G, float eps, float *g_out)
+{
+    orc_pool PK = {k_pages, num_pages, page_size, n_kv_heads, head_dim};
+    orc_pool PV = {v_pages, num_pages, page_size, n_kv_heads, head_dim};
+    const int D = head_dim;
+    if (T < 1 || G < 1) return -1;
+    double *a = (double *)calloc((size_t)T, sizeof(double));
+    double *l = (double *)malloc(sizeof(double) * (size_t)T);
+    double *kd = (double *)malloc(sizeof(double) * (size_t)D);
+    if (!a || !l || !kd) { free(a); free(l); free(kd); return -2; }
+    for (int r = 0; r < G; ++r) {
+        const float *mu = mean + (int64_t)r * D;
+        const uint16_t *S = cov + (int64_t)r * D * D;
+        double mx = -INFINITY;
+        for (int t = 0; t < T; ++t) {
+            const uint16_t *kt = k_row(&PK, layer, table_row, t, h);
+            for (int j = 0; j < D; ++j) kd[j] = bf16_to_double(kt[j]);
+            double lin = 0.0, quad = 0.0;
+            for (int j = 0; j < D; ++j) {
+                lin += (double)mu[j] * kd[j];
+                double sk = 0.0; /* (Sigma k)_j */
+                for (int i = 0; i < D; ++i) sk += bf16_to_double(S[(int64_t)j * D + i]) * kd[i];
+                quad += kd[j] * sk;
+            }
+            l[t] = lin / sqrt((double)D) + quad / (2.0 * (double)D);
+            if (l[t] > mx) mx = l[t];
+        }
+        double Z = 0.0;
+        for (int t = 0; t < T; ++t) { l[t] = exp(l[t] - mx); Z += l[t]; }
+        for (int t = 0; t < T; ++t) a[t] += l[t] / Z;
+    }
+    for (int t = 0; t < T; ++t) {
+        const uint16_t *vt = v_row(&PV, layer, table_row, t, h);
+        double v2 = 0.0;
+        for (int j = 0; j < D; ++j) { const double x = bf16_to_double(vt[j]); v2 += x * x; }
+        g_out[t] = (float)((a[t] / (double)G + (double)eps) * sqrt(v2));
+    }
+    free(a); free(l); free(kd);
     return 0;
 }
 

@@ -18,6 +18,10 @@ Recipe (per layer, seed = 260523200 + 10^6*config + 10^3*step + layer):
     direction; then 1 % of positions (all heads) scaled by 3;
   * queries ~ N(0,1) + 2 * direction of their KV head; values ~ N(0,1);
   * appended tokens: same, without spans;
+  * query statistics for the expected-attention scorer (the mean and covariance a runtime
+    would estimate from recent queries): mean = 2 * direction + 0.1 * N(0,1); covariance =
+    0.5 I + sum of eight rank-one terms lambda_i u_i u_i^T, u_0 the direction, the other u_i
+    random unit vectors, lambda_i uniform in [0.5, 4]; rounded to bf16;
   * pages drawn from a seeded random permutation of the pool.
 """
 from __future__ import annotations
@@ -31,7 +35,7 @@ SEED_BASE = 260523200
 PAGE = 16
 HEAD_DIM = 128
 
-SCORER_TOVA, SCORER_KEYDIFF, SCORER_EXTERNAL = 0, 1, 2
+SCORER_TOVA, SCORER_KEYDIFF, SCORER_EXTERNAL, SCORER_EXPECTED = 0, 1, 2, 3
 
 
 @dataclass(frozen=True)
@@ -179,6 +183,28 @@ def _make_queries(wl: Workload, step: int, directions: torch.Tensor, device) -> 
         d = directions[l].repeat_interleave(wl.group, dim=0)  # [Hq][128]
         q[l] = (x + 2.0 * d[None, :, None, :]).to(torch.bfloat16)
     return q
+
+
+def make_query_stats(cache: "Cache"):
+    """Mean (fp32 [L][B][Hq][128]) and covariance (bf16 [L][B][Hq][128][128]) of the future queries of every
+    query head, as a serving runtime would estimate them; seeded by configuration, step and layer."""
+    wl = cache.wl
+    device = cache.k_pages.device
+    L, B, Hq = wl.layers_resident, wl.batch, wl.n_q_heads
+    mean = torch.empty((L, B, Hq, HEAD_DIM), device=device, dtype=torch.float32)
+    cov = torch.empty((L, B, Hq, HEAD_DIM, HEAD_DIM), device=device, dtype=torch.bfloat16)
+    eye = torch.eye(HEAD_DIM, device=device)
+    for l in range(L):
+        gen = _gen(device, _seed(wl.cfg_id, cache.step, l) + 700)
+        d = cache.directions[l].repeat_interleave(wl.group, dim=0)  # [Hq][128]
+        mean[l] = 2.0 * d[None] + 0.1 * torch.randn((B, Hq, HEAD_DIM), generator=gen, device=device)
+        u = torch.randn((B, Hq, 8, HEAD_DIM), generator=gen, device=device)
+        u = u / u.norm(dim=-1, keepdim=True)
+        u[:, :, 0] = d[None]
+        lam = 0.5 + 3.5 * torch.rand((B, Hq, 8), generator=gen, device=device)
+        c = 0.5 * eye + torch.einsum("bhr,bhri,bhrj->bhij", lam, u, u)
+        cov[l] = c.to(torch.bfloat16)
+    return mean, cov
 
 
 def make_cache(wl: Workload, device="cpu", shuffle_pages: bool = True) -> Cache:

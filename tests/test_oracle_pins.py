@@ -602,6 +602,95 @@ def test_keydiff_is_negative_cosine_to_mean_key():
     assert g[4] > 0.9 and g[0] < -0.9
 
 
+def _u16(t):
+    return t.to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+
+
+def _expected_logits(K, mean, cov):
+    """l_t = mu.k_t / sqrt(D) + k_t^T Sigma k_t / (2 D), by library matrix products in fp64."""
+    D = K.shape[1]
+    return K @ mean / np.sqrt(D) + ((K @ cov) * K).sum(1) / (2 * D)
+
+
+def test_expected_attention_is_the_gaussian_expectation_of_the_attention_weight():
+    """The logit the scorer exponentiates is log E[exp(q.k / sqrt(D))] for q ~ N(mu, Sigma) (the idea the paper's
+    expected-attention scorer is named for): checked against a Monte-Carlo mean over sampled queries, which knows
+    nothing of the closed form.  With uniform values the score is softmax(logit) + eps times the value norm."""
+    rng = np.random.default_rng(31)
+    T, D = 48, 128
+    pages_k, table, dense = _tiny_cache(rng, T=T, P=4, H=1)
+    K = dense[0, :, 0].numpy() * 0.5
+    pages_k = _u16(torch.from_numpy(pages_k.view(np.int16)).view(torch.bfloat16).float() * 0.5)   # keys halved: tame variance
+    A = rng.standard_normal((D, 6)) * 0.6
+    cov = torch.from_numpy(A @ A.T + 0.25 * np.eye(D)).to(torch.bfloat16)
+    mean = rng.standard_normal(D).astype(np.float32) * 0.5
+    cov64 = cov.double().numpy()
+    # values: every row the same vector of norm 5 (3, 4, 0, ...)
+    v = torch.zeros((1, 4, 16, 1, D)); v[..., 0] = 3.0; v[..., 1] = 4.0
+    eps = 0.01
+    g = oracle.score_expected(pages_k, _u16(v), 0, 0, table, T, mean[None], _u16(cov)[None], eps)
+    # Monte Carlo: q = mu + C z with C C^T = Sigma (Sigma as the scorer reads it, after rounding to bf16, symmetrised)
+    sym = (cov64 + cov64.T) / 2
+    w, U = np.linalg.eigh(sym)
+    C = U * np.sqrt(np.clip(w, 0, None))
+    n = 400_000
+    z = rng.standard_normal((n, D))
+    q = mean.astype(np.float64) + z @ C.T
+    mc = np.exp(q @ K.T / np.sqrt(D))                    # [n][T]
+    est, se = mc.mean(0), mc.std(0) / np.sqrt(n)
+    closed = np.exp(_expected_logits(K, mean.astype(np.float64), sym))
+    assert (np.abs(est - closed) < 6 * se + 1e-12).all()
+    assert (se / closed < 0.02).all()                    # (the estimate is sharp enough to tell 1/2 from 1 in the quadratic term)
+    ref = (closed / closed.sum() + eps) * 5.0
+    np.testing.assert_allclose(g, ref, rtol=2e-6)
+
+
+def test_expected_attention_special_cases():
+    rng = np.random.default_rng(32)
+    T, D, H = 150, 128, 2
+    pages_k, table, dense = _tiny_cache(rng, T=T, P=12, H=H)
+    pages_v, _, dense_v = _tiny_cache(np.random.default_rng(33), T=T, P=12, H=H)
+    slots = table[np.arange(T) // 16] * 16 + np.arange(T) % 16
+    V = torch.from_numpy(pages_v.view(np.int16)).view(torch.bfloat16).double().reshape(1, -1, H, D)[0, slots]   # values through this cache's table
+    h = 1
+    K = dense[0, :, h].numpy()
+    vnorm = V[:, h].norm(dim=1).numpy()
+    mu = torch.from_numpy(rng.standard_normal(D).astype(np.float32)).to(torch.bfloat16)
+    zero = np.zeros((1, D, D), np.uint16)
+    # zero covariance: the softmax of one query, i.e. the TOVA score of the query mu (another routine of the oracle,
+    # itself pinned to the library softmax), times the value norm
+    g0 = oracle.score_expected(pages_k, pages_v, 0, h, table, T, mu.float().numpy()[None], zero, 0.0)
+    u = oracle.score_tova(pages_k, 0, h, table, T, _u16(mu).reshape(1, 1, D), 1, 1, False)
+    np.testing.assert_allclose(g0, u.astype(np.float64) * vnorm, rtol=3e-6)
+    # eps is added before the value norm multiplies
+    g1 = oracle.score_expected(pages_k, pages_v, 0, h, table, T, mu.float().numpy()[None], zero, 0.25)
+    np.testing.assert_allclose(g1, (u.astype(np.float64) + 0.25) * vnorm, rtol=3e-6)
+    # isotropic covariance s^2 I: logit = mu.k / sqrt(D) + s^2 |k|^2 / (2 D)
+    s2 = 0.75
+    iso = _u16(torch.eye(D) * s2)[None]
+    g2 = oracle.score_expected(pages_k, pages_v, 0, h, table, T, mu.float().numpy()[None], iso, 0.0)
+    lg = K @ mu.double().numpy() / np.sqrt(D) + s2 * (K * K).sum(1) / (2 * D)
+    ref = np.exp(lg - lg.max()); ref /= ref.sum()
+    np.testing.assert_allclose(g2, ref * vnorm, rtol=3e-6)
+    # a general covariance against library matrix products; only its symmetric part matters
+    Cm = torch.from_numpy(rng.standard_normal((D, D)) * 0.05).to(torch.bfloat16)
+    g3 = oracle.score_expected(pages_k, pages_v, 0, h, table, T, mu.float().numpy()[None], _u16(Cm)[None], 0.0)
+    lg = _expected_logits(K, mu.double().numpy(), Cm.double().numpy())
+    ref = np.exp(lg - lg.max()); ref /= ref.sum()
+    np.testing.assert_allclose(g3, ref * vnorm, rtol=3e-6)
+    g3t = oracle.score_expected(pages_k, pages_v, 0, h, table, T, mu.float().numpy()[None], _u16(Cm.T.contiguous())[None], 0.0)
+    np.testing.assert_allclose(g3t, g3, rtol=1e-6)
+    # group: the mean of the heads' softmaxes (not a softmax of mean logits); identical heads collapse
+    mu_b = torch.from_numpy(rng.standard_normal(D).astype(np.float32) * 3).to(torch.bfloat16)
+    gg = oracle.score_expected(pages_k, pages_v, 0, h, table, T, np.stack([mu.float().numpy(), mu_b.float().numpy()]),
+                               np.concatenate([iso, zero]), 0.0)
+    ub = oracle.score_tova(pages_k, 0, h, table, T, _u16(mu_b).reshape(1, 1, D), 1, 1, False)
+    np.testing.assert_allclose(gg, (g2 / vnorm + ub) / 2 * vnorm, rtol=5e-6)
+    same = oracle.score_expected(pages_k, pages_v, 0, h, table, T, np.stack([mu.float().numpy()] * 3),
+                                 np.concatenate([iso] * 3), 0.0)
+    np.testing.assert_allclose(same, g2, rtol=1e-6)
+
+
 # ----------------------------------------------------------------------------- usage smoothing, decoupled signals
 
 def test_usage_smoothing_hand_computed_and_library_pooling():
@@ -671,6 +760,17 @@ def test_smoothing_changes_the_mass_only_and_decoupled_signals_split_roles():
             a, b = r.bounds[i], r.bounds[i + 1]
             order = sorted(range(a, b), key=lambda t: (-g[t], t))[: r.quotas[i]]
             assert set(order) <= set(r.keep_idx.tolist())
+    # the expected-attention scorer as base score: alone (u = g) and with the window attention as the mass signal
+    stats = dict(q_mean=rng.standard_normal((1, 1, 4, 128)).astype(np.float32),
+                 q_cov=_u16(torch.from_numpy(rng.standard_normal((1, 1, 4, 128, 128)) * 0.05)), score_eps=0.01)
+    ex = run(scorer=oracle.SCORER_EXPECTED, **stats)
+    exd = run(scorer=oracle.SCORER_EXPECTED, decoupled=True, **stats)
+    for (l, b, h) in base:
+        want = oracle.score_expected(pages, pages, l, h, tab[b], T, stats["q_mean"][l, b, 2 * h:2 * h + 2],
+                                     stats["q_cov"][l, b, 2 * h:2 * h + 2], 0.01)
+        assert (ex[(l, b, h)].scores == want).all() and (ex[(l, b, h)].usage == want).all()
+        assert (exd[(l, b, h)].scores == want).all() and (exd[(l, b, h)].usage == base[(l, b, h)].scores).all()
+        assert (exd[(l, b, h)].bounds == base[(l, b, h)].bounds).all()
     # an external usage signal plays the same role
     ext_g = rng.standard_normal((1, 1, 2, T)).astype(np.float32)
     ext_u = np.exp(rng.standard_normal((1, 1, 2, T))).astype(np.float32)
