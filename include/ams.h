@@ -9,8 +9,8 @@
  * Algorithm 1 of the paper followed by the paged head-wise compaction of its
  * serving appendix:
  *   1. score every cached token (TOVA-style observation-window softmax averaged
- *      over the GQA group — Section 3.2 and Algorithm 1 step 1 — or a key-only
- *      KeyDiff-style score);
+ *      over the GQA group — Section 3.2 and Algorithm 1 step 1 — a key-only
+ *      KeyDiff-style score, or the expected-attention score of ams_set_query_stats);
  *   2. turn usage into the normalised quality mass (Eq. 1), mix it with the EMA
  *      credit carried across events (Section 3.3, "EMA credit"; Algorithm 1 step 2);
  *   3. prefix-sum the mass, cut at multiples of the segment mass, merge short and
@@ -71,7 +71,7 @@ enum {
     AMS_ERR_INTERNAL = -6     /* a device-side consistency check failed                       */
 };
 
-enum { AMS_SCORER_TOVA = 0, AMS_SCORER_KEYDIFF = 1, AMS_SCORER_EXTERNAL = 2 };
+enum { AMS_SCORER_TOVA = 0, AMS_SCORER_KEYDIFF = 1, AMS_SCORER_EXTERNAL = 2, AMS_SCORER_EXPECTED = 3 };
 
 typedef struct ams_state ams_state; /* opaque host handle */
 
@@ -101,6 +101,8 @@ typedef struct {
                                                 mass quantile; merge and split as usual       */
     int32_t uniform_quotas;                  /* 1: component ablation "w/o mass-weighted quotas":
                                                 the budget is shared by segment length        */
+    int32_t expected_scorer;                 /* 1: reserve room for AMS_SCORER_EXPECTED (one fp32
+                                                logit per query head and cached token)        */
 } ams_config;
 
 /* Optional device outputs for inspection and tests; any member may be NULL.
@@ -148,7 +150,7 @@ int ams_init_state(const ams_config *cfg, void *ema_state, void *workspace, size
  *  block_table, seq_lens : updated in place for every sequence with seq_len > budget:
  *                     row <- dst_pages row followed by -1, length <- budget.  Sequences with
  *                     seq_len <= budget are left as they are (nothing to evict).
- *  obs_queries, window : may be NULL / 0 for AMS_SCORER_KEYDIFF and AMS_SCORER_EXTERNAL.
+ *  obs_queries, window : may be NULL / 0 for AMS_SCORER_KEYDIFF, AMS_SCORER_EXPECTED and AMS_SCORER_EXTERNAL.
  *  ema_state        : the buffer given to ams_init_state (or a restored copy of it).
  *  n_segments       : S, the number of mass quantiles (segment mass 1/S), 1..max_segments.
  *  ext_scores       : AMS_SCORER_EXTERNAL only: fp32 [L][batch][H][max_seq_len] (16-byte aligned) base
@@ -157,9 +159,9 @@ int ams_init_state(const ams_config *cfg, void *ema_state, void *workspace, size
  *                     the usage u.
  * Mass signal (Algorithm 1 step 1; the runtime section's "decoupled mass and selection scores"):
  * the mass is built from the usage u, tokens inside a segment are ranked by the base score g.
- * By default u = g = the scorer's output.  With cfg.decoupled = 1, AMS_SCORER_KEYDIFF and
- * observation queries given (obs_queries != NULL, window >= 1), u is the window attention of
- * AMS_SCORER_TOVA and g the key-only score.  cfg.pool_kernel = k > 1 replaces u (never g) by its
+ * By default u = g = the scorer's output.  With cfg.decoupled = 1, AMS_SCORER_KEYDIFF or
+ * AMS_SCORER_EXPECTED and observation queries given (obs_queries != NULL, window >= 1), u is the
+ * window attention of AMS_SCORER_TOVA and g the scorer's own score.  cfg.pool_kernel = k > 1 replaces u (never g) by its
  * zero-padded average over k neighbouring positions: u'_t = (sum of u_j, |j - t| <= k/2, j inside
  * the sequence, added left to right in fp32) / k.
  *  dbg              : optional views, or NULL.
@@ -173,6 +175,23 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
                  int32_t window, void *ema_state, int32_t budget, int32_t n_segments, int32_t scorer_id,
                  const int32_t *dst_pages, const float *ext_scores, const float *ext_usage,
                  const ams_debug_views *dbg, void *stream);
+
+/* Query statistics for AMS_SCORER_EXPECTED, the expected-attention scorer behind the paper's
+ * "AMS-Expected" rows (experimental-setup section and the baseline table of the appendix name it and
+ * its regularisation coefficient 1e-2; the formula is the closed form of the work they cite, for
+ * queries modelled as Gaussian).  For query head r of a KV head's group and cached token t:
+ *     l_{r,t} = mu_r . k_t / sqrt(128) + k_t^T Sigma_r k_t / (2 * 128)
+ *     score_t = (mean over r of softmax_t(l_{r,.}) + score_eps) * |v_t|_2
+ *   q_mean : DEVICE fp32 [n_layers][batch][n_q_heads][128], 16-byte aligned
+ *   q_cov  : DEVICE bf16 [n_layers][batch][n_q_heads][128][128] (row-major; only the symmetric part matters),
+ *            16-byte aligned
+ * `batch` is that of the ams_compress calls that follow.  The pointers are kept in the handle and read by
+ * every later ams_compress with AMS_SCORER_EXPECTED (the buffers stay the caller's and must stay valid);
+ * estimating them from the model's recent queries is the caller's job.  cfg.expected_scorer must be 1.
+ * With cfg.decoupled = 1 and observation queries given, the mass comes from the window attention and
+ * this score ranks the tokens inside the segments (the runtime section's "decoupled mass and selection
+ * scores, including TOVA-style and expected-attention selection"). */
+int ams_set_query_stats(ams_state *st, const float *q_mean, const void *q_cov, float score_eps);
 
 /* Synchronises `stream`, then returns and clears the device status: AMS_OK or the
  * first device-side error.  detail[0..3] (host, may be NULL) receive the code, the

@@ -20,12 +20,12 @@ LIB_PATH = os.path.join(_HERE, "libams.so")
 AMS_OK = 0
 AMS_ERR_INVALID_ARG, AMS_ERR_UNSUPPORTED, AMS_ERR_CAPACITY = -1, -2, -3
 AMS_ERR_CUDA, AMS_ERR_TIMEOUT, AMS_ERR_INTERNAL = -4, -5, -6
-AMS_SCORER_TOVA, AMS_SCORER_KEYDIFF, AMS_SCORER_EXTERNAL = 0, 1, 2
+AMS_SCORER_TOVA, AMS_SCORER_KEYDIFF, AMS_SCORER_EXTERNAL, AMS_SCORER_EXPECTED = 0, 1, 2, 3
 
 EXPORTS = ["ams_config_default", "ams_ema_state_bytes", "ams_workspace_bytes", "ams_segment_capacity",
            "ams_init_state", "ams_compress", "ams_get_status", "ams_last_launch_count", "ams_free",
            "ams_strerror", "ams_set_profiling", "ams_get_kernel_times", "ams_kernel_name", "ams_select_static",
-           "ams_select_static_status", "ams_debug_expire_wait"]
+           "ams_select_static_status", "ams_debug_expire_wait", "ams_set_query_stats"]
 KERNEL_SLOTS = 10
 
 
@@ -35,7 +35,7 @@ class AmsConfig(ctypes.Structure):
                  "max_window", "max_budget", "max_segments", "l_min", "l_max", "q_min", "n_sink", "n_last")] + \
                [("ema_lambda", ctypes.c_float), ("ema_beta", ctypes.c_float), ("eps", ctypes.c_float),
                 ("causal_window", ctypes.c_int32), ("pool_kernel", ctypes.c_int32), ("decoupled", ctypes.c_int32),
-                ("fixed_segments", ctypes.c_int32), ("uniform_quotas", ctypes.c_int32)]
+                ("fixed_segments", ctypes.c_int32), ("uniform_quotas", ctypes.c_int32), ("expected_scorer", ctypes.c_int32)]
 
 
 class AmsDebugViews(ctypes.Structure):
@@ -89,6 +89,8 @@ def lib() -> ctypes.CDLL:
         L.ams_select_static_status.restype = ctypes.c_int
         L.ams_debug_expire_wait.argtypes = [ctypes.c_void_p, ctypes.c_uint32, ctypes.c_void_p]
         L.ams_debug_expire_wait.restype = ctypes.c_int
+        L.ams_set_query_stats.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_float]
+        L.ams_set_query_stats.restype = ctypes.c_int
         L.ams_strerror.argtypes = [ctypes.c_int]
         L.ams_strerror.restype = ctypes.c_char_p
         _lib = L
@@ -195,6 +197,16 @@ class AmsCompressor:
         if rc != AMS_OK:
             raise AmsError(rc, "ams_compress")
 
+    def set_query_stats(self, q_mean: torch.Tensor, q_cov: torch.Tensor, score_eps: float = 1e-2) -> None:
+        """Mean (fp32 [L][batch][Hq][128]) and covariance (bf16 [L][batch][Hq][128][128]) of the future queries for
+        AMS_SCORER_EXPECTED; the tensors are kept alive by this object until they are replaced."""
+        assert q_mean.dtype == torch.float32 and q_mean.is_contiguous() and q_mean.shape[-1] == 128
+        assert q_cov.dtype == torch.bfloat16 and q_cov.is_contiguous() and q_cov.shape == q_mean.shape + (128,)
+        rc = lib().ams_set_query_stats(self._h, _ptr(q_mean), _ptr(q_cov), ctypes.c_float(score_eps))
+        if rc != AMS_OK:
+            raise AmsError(rc, "ams_set_query_stats")
+        self._query_stats = (q_mean, q_cov)
+
     def status(self, stream: torch.cuda.Stream | None = None, check: bool = True):
         s = stream or torch.cuda.current_stream(self.device)
         detail = (ctypes.c_int32 * 4)()
@@ -270,4 +282,4 @@ def config_for(wl, **kw) -> AmsConfig:
                           q_min=wl.q_min, n_sink=wl.n_sink, n_last=wl.n_last, ema_lambda=wl.ema_lambda,
                           ema_beta=wl.ema_beta, eps=wl.eps, pool_kernel=wl.pool_kernel, decoupled=int(wl.decoupled),
                           fixed_segments=int(wl.fixed_segments), uniform_quotas=int(wl.uniform_quotas),
-                          **kw)
+                          **{"expected_scorer": int(wl.scorer_id == AMS_SCORER_EXPECTED), **kw})

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libams.so")
-SOURCES = ["ams_api.cu", "ams_score.cu", "ams_score_tc.cu", "ams_segment.cu", "ams_segsel.cu", "ams_gather.cu", "ams_usage.cu"]
+SOURCES = ["ams_api.cu", "ams_score.cu", "ams_score_tc.cu", "ams_score_expected.cu", "ams_segment.cu", "ams_segsel.cu", "ams_gather.cu", "ams_usage.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC"]
 

@@ -8,7 +8,7 @@
 namespace ams {
 
 struct Layout {
-    size_t status, eff_lens, seq_bad, scores, usage, logits, cbuf, n_seg, raw_cuts, seg_bounds, quotas, keep_idx, part, fin, total;
+    size_t status, eff_lens, seq_bad, scores, usage, logits, ex_logits, cbuf, n_seg, raw_cuts, seg_bounds, quotas, keep_idx, part, fin, total;
     int units, T_cap, seg_cap, n_slices, slice_len, rows_pad_cap;
 };
 
@@ -29,6 +29,7 @@ static bool config_ok(const ams_config *c, int *why)
     if (c->pool_kernel < 1 || c->pool_kernel > 63 || !(c->pool_kernel & 1)) return false;
     if (c->decoupled != 0 && c->decoupled != 1) return false;
     if ((c->fixed_segments != 0 && c->fixed_segments != 1) || (c->uniform_quotas != 0 && c->uniform_quotas != 1)) return false;
+    if (c->expected_scorer != 0 && c->expected_scorer != 1) return false;
     *why = AMS_ERR_UNSUPPORTED;
     if (c->head_dim != kHeadDim || c->page_size != kPage) return false;
     if (c->n_q_heads % c->n_kv_heads) return false;
@@ -101,6 +102,8 @@ static Layout make_layout(const ams_config *c)
     // narrow query blocks keep their logits (rows_pad floats per token, at most 1/4 of the K bytes) so that
     // the usage pass need not read K again
     y.logits = off;     off = align_up(off + (y.rows_pad_cap <= 16 && c->max_window > 0 ? U * T * (size_t)y.rows_pad_cap * 4 : 0), 256);
+    // expected-attention scorer: one logit per (query head, token), so that K is read once
+    y.ex_logits = off;  off = align_up(off + (c->expected_scorer ? U * T * (size_t)(c->n_q_heads / c->n_kv_heads) * 4 : 0), 256);
     y.total = off;
     return y;
 }
@@ -116,6 +119,9 @@ struct ams_state {
     void *ema;
     int32_t last_launches;
     cudaEvent_t ev[32];
+    const float *q_mean; // query statistics of the expected-attention scorer (ams_set_query_stats)
+    const void *q_cov;
+    float score_eps;
     bool profiling;
     int n_ev;
     int ev_ids[32];
@@ -143,6 +149,7 @@ void ams_config_default(ams_config *cfg)
     cfg->decoupled = 0;
     cfg->fixed_segments = 0;
     cfg->uniform_quotas = 0;
+    cfg->expected_scorer = 0;
 }
 
 size_t ams_ema_state_bytes(const ams_config *cfg)
@@ -190,6 +197,9 @@ int ams_init_state(const ams_config *cfg, void *ema_state, void *workspace, size
     st->ws = (unsigned char *)workspace;
     st->ema = ema_state;
     st->last_launches = 0;
+    st->q_mean = nullptr;
+    st->q_cov = nullptr;
+    st->score_eps = 0.0f;
     st->profiling = false;
     st->n_ev = 0;
     *out = st;
@@ -212,12 +222,15 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
         if (!obs_queries || window < 1 || window > c.max_window) return AMS_ERR_INVALID_ARG;
     } else if (scorer_id == AMS_SCORER_EXTERNAL) {
         if (!ext_scores) return AMS_ERR_INVALID_ARG;
+    } else if (scorer_id == AMS_SCORER_EXPECTED) {
+        if (!c.expected_scorer) return AMS_ERR_CAPACITY; // no room was reserved for the logits
+        if (!st->q_mean || !st->q_cov) return AMS_ERR_INVALID_ARG;
     } else if (scorer_id != AMS_SCORER_KEYDIFF) {
         return AMS_ERR_INVALID_ARG;
     }
     if (ext_usage && scorer_id != AMS_SCORER_EXTERNAL) return AMS_ERR_INVALID_ARG;
     // key-only base scores with the window attention as mass signal
-    const bool split = scorer_id == AMS_SCORER_KEYDIFF && c.decoupled && obs_queries && window >= 1;
+    const bool split = (scorer_id == AMS_SCORER_KEYDIFF || scorer_id == AMS_SCORER_EXPECTED) && c.decoupled && obs_queries && window >= 1;
     if (split && window > c.max_window) return AMS_ERR_INVALID_ARG;
     if (((uintptr_t)k_pages | (uintptr_t)v_pages | (uintptr_t)obs_queries | (uintptr_t)ema_state | (uintptr_t)ext_scores |
          (uintptr_t)ext_usage) & 15) return AMS_ERR_INVALID_ARG;
@@ -258,6 +271,8 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
     p.tc_stages = p.rows_pad <= 256 ? 4 : 2; // even: each stage then belongs to one of the two MMA issuers
     p.status = (int *)(st->ws + y.status);
     p.logits = (y.rows_pad_cap <= 16 && c.max_window > 0) ? (float *)(st->ws + y.logits) : nullptr;
+    p.q_mean = st->q_mean; p.q_cov = (const __nv_bfloat16 *)st->q_cov; p.score_eps = st->score_eps;
+    p.ex_logits = c.expected_scorer ? (float *)(st->ws + y.ex_logits) : nullptr;
 
     int rc = AMS_OK;
     LaunchCtx ctx;
@@ -271,7 +286,7 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
     p.W = scorer_id == AMS_SCORER_TOVA ? window : 0;
     if (rc == AMS_OK && scorer_id == AMS_SCORER_TOVA) {
         rc = launch_score_tova(p, ctx);
-    } else if (rc == AMS_OK && scorer_id == AMS_SCORER_KEYDIFF) {
+    } else if (rc == AMS_OK && (scorer_id == AMS_SCORER_KEYDIFF || scorer_id == AMS_SCORER_EXPECTED)) {
         if (split) {
             // the window attention goes through the score array into the usage array (smoothed on the way
             // if asked for); the key-only score then takes the score array
@@ -284,7 +299,7 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
             if (rc == AMS_OK) rc = launch_smooth_usage(p, p.scores, usage_buf, c.pool_kernel, ctx);
             p.usage = usage_buf;
         }
-        if (rc == AMS_OK) rc = launch_score_keydiff(p, ctx);
+        if (rc == AMS_OK) rc = scorer_id == AMS_SCORER_KEYDIFF ? launch_score_keydiff(p, ctx) : launch_score_expected(p, ctx);
     }
     if (rc == AMS_OK && c.pool_kernel > 1 && !split) {
         rc = launch_smooth_usage(p, p.usage, usage_buf, c.pool_kernel, ctx);
@@ -309,6 +324,16 @@ int ams_compress(ams_state *st, void *k_pages, void *v_pages, int64_t num_pages,
     st->n_ev = ctx.n_ev;
     memcpy(st->ev_ids, ctx.ids, sizeof ctx.ids);
     return rc;
+}
+
+int ams_set_query_stats(ams_state *st, const float *q_mean, const void *q_cov, float score_eps)
+{
+    if (!st || !q_mean || !q_cov || !(score_eps >= 0.0f) || !(score_eps < 1e30f)) return AMS_ERR_INVALID_ARG;
+    if (((uintptr_t)q_mean | (uintptr_t)q_cov) & 15) return AMS_ERR_INVALID_ARG;
+    st->q_mean = q_mean;
+    st->q_cov = q_cov;
+    st->score_eps = score_eps;
+    return AMS_OK;
 }
 
 int ams_get_status(ams_state *st, void *stream, int32_t *detail)

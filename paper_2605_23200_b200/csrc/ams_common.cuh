@@ -54,6 +54,12 @@ struct DevParams {
     int tc_tpc_min, tc_stages;        // tensor-core scorer: least tiles per block, K stages in shared memory
     int tc_hpb;                       // tensor-core scorer: KV heads a block takes one after the other (set by its launcher)
     float *logits;                    // narrow query blocks (rows_pad <= 16): scaled logits [units][T_cap][rows_pad], or null
+    // expected-attention scorer
+    const float *q_mean;              // [L][B][H*G][128] mean of the future queries per query head
+    const __nv_bfloat16 *q_cov;       // [L][B][H*G][128][128] their covariance
+    float score_eps;                  // added to the group-mean attention weight before the value norm multiplies
+    float *ex_logits;                 // [units][G][T_cap] logits in log2 units, or null
+    int ex_g0, ex_gc;                 // query heads [g0, g0 + gc) of the group handled by one launch (set by the launcher)
     int *seq_bad;                     // [B]: set when a unit of the sequence reported a device-side error (its rows stay)
     int *status;                      // [4]: code, unit, a, b
 };
@@ -164,6 +170,26 @@ __device__ __forceinline__ unsigned score_key(float x)
 __device__ __forceinline__ float bf16_lo(unsigned w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(unsigned w) { return __uint_as_float(w & 0xffff0000u); }
 
+// Packed fp32 pairs (two floats in a 64-bit register) and their fused multiply-add.
+__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi)
+{
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ unsigned long long fma_f32x2(unsigned long long a, unsigned long long b, unsigned long long c)
+{
+    unsigned long long r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ float sum_f32x2(unsigned long long a)
+{
+    float lo, hi;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(a));
+    return lo + hi;
+}
+
 // 16-byte global load that does not pollute L1 (streamed once per phase).
 __device__ __forceinline__ uint4 ld_stream16(const void *ptr)
 {
@@ -231,6 +257,8 @@ bool tova_tc_supported(const DevParams &p);
 size_t tova_tc_smem_bytes(const DevParams &p);
 int launch_score_tova_tc(const DevParams &p, LaunchCtx &ctx);
 int launch_score_keydiff(const DevParams &p, LaunchCtx &ctx);
+bool expected_supported(const DevParams &p);
+int launch_score_expected(const DevParams &p, LaunchCtx &ctx);
 bool segsel_supported(const DevParams &p);   // shared-memory need of the selection kernels fits (always, within the configuration limits)
 int launch_segsel(const DevParams &p, LaunchCtx &ctx); // Algorithm 1 steps 1-5: three kernels
 int launch_gather(const DevParams &p, LaunchCtx &ctx);

@@ -275,26 +275,6 @@ __global__ void __launch_bounds__(256) k_tova_usage_from_logits(DevParams p)
 
 constexpr int kKdThreads = 256; // 16 token rows x 16 lanes of 16 bytes
 
-// Packed fp32 pairs (two floats in a 64-bit register) and their fused multiply-add.
-__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi)
-{
-    unsigned long long r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ unsigned long long fma_f32x2(unsigned long long a, unsigned long long b, unsigned long long c)
-{
-    unsigned long long r;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-    return r;
-}
-__device__ __forceinline__ float sum_f32x2(unsigned long long a)
-{
-    float lo, hi;
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(a));
-    return lo + hi;
-}
-
 __global__ void __launch_bounds__(kKdThreads) k_keydiff_sum(DevParams p)
 {
     __shared__ float red[16][kHeadDim];

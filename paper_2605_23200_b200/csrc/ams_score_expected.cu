@@ -1,0 +1,429 @@
+// Expected-attention scorer on the sm_100a tensor path.  For every query head r of a KV head's GQA
+// group the caller gives the mean mu_r and the covariance Sigma_r of the head's future queries; the
+// expected attention weight of key k_t under q ~ N(mu_r, Sigma_r) is exp(l_{r,t}) with
+//     l_{r,t} = mu_r . k_t / sqrt(d) + k_t^T Sigma_r k_t / (2 d),
+// and the score is (mean_r softmax_t(l_{r,.}) + eps) * |v_t|.
+//
+// k_expected_tc reads K once: a 128-token tile is the A operand (tokens on the TMEM lanes) and the
+// group's covariance matrices, resident in shared memory, are the B operands, so that one
+// tcgen05.mma chain per head leaves (Sigma_r k_t) of token t in the 128 columns of TMEM lane t.  The
+// thread that owns the lane dots them with k_t (read from the same shared-memory tile) and with mu_r,
+// stores the logit and keeps a running (max, sum of 2^x) per head.  The block shape and the pipeline are those of
+// the window scorer: warp 0 feeds K tiles by TMA, warps 1 and 3 issue the MMAs for the two consumer
+// pairs, warps 4-19 are four consumer warpgroups (two per tile, each taking 64 of a head's 128
+// columns).  k_expected_final then streams V and the stored logits (16 bytes per token and head
+// group of four) and writes the scores.  Every wait is bounded; on expiry the block reports
+// AMS_ERR_TIMEOUT, drains its copies, frees its TMEM and returns.
+#include <cuda.h>
+
+#include "ams_common.cuh"
+#include "ams_tc_ptx.cuh"
+#include "ams_tc_tiles.cuh"
+
+namespace ams {
+
+using namespace tc;
+
+namespace {
+
+constexpr int kExHeads = 4; // query heads per launch: 4 x 128 accumulator columns are the whole TMEM
+
+struct ExShared {
+    unsigned long long kfull[kMaxStages], kempty[kMaxStages], tfull[kSlots], tempty[kSlots];
+    unsigned long long cfull, cempty, done[2];
+    unsigned long long pfull[2][2];  // the second half's part of a logit is in pacc[pair][slot bit]
+    float pacc[2][2][128];
+    float2 red[8][kExHeads];         // per first-half consumer warp and head: (max, sum of 2^(x - max))
+    float2 stat[kExHeads][256];      // running (max, sum) of every first-half consumer thread, per head
+    uint32_t tmem_base;
+    int abort_flag;
+    int tiles_lh, tpc;
+    long long n_tiles;
+};
+
+__global__ void __launch_bounds__(kTcThreads, 1) k_expected_tc(DevParams p, const __grid_constant__ CUtensorMap k_map,
+                                                               const __grid_constant__ CUtensorMap c_map)
+{
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    __shared__ ExShared sh;
+    __shared__ int prefix[1025];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n_rb = p.ex_gc, NS = p.tc_stages; // one 128-column accumulator block per query head
+    unsigned char *base = reinterpret_cast<unsigned char *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    unsigned char *Cs = base;                                   // [n_rb][2 halves][128 rows][128 B]
+    unsigned char *Ks = Cs + (size_t)n_rb * kTileBytes;         // [NS][8-row group][2 halves][8 rows][128 B]
+    float *mu_s = reinterpret_cast<float *>(Ks + (size_t)NS * kTileBytes); // [2][n_rb][128], scaled
+    volatile int *abort_flag = &sh.abort_flag;
+
+    if (tid == 0) {
+        for (int i = 0; i < kMaxStages; ++i) {
+            mbar_init(smem_u32(&sh.kfull[i]), 1);
+            mbar_init(smem_u32(&sh.kempty[i]), 9); // the issuer's commit and the eight consumer warps that read the rows
+        }
+        for (int i = 0; i < kSlots; ++i) { mbar_init(smem_u32(&sh.tfull[i]), 1); mbar_init(smem_u32(&sh.tempty[i]), 8); }
+        for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&sh.pfull[i >> 1][i & 1]), 4);
+        mbar_init(smem_u32(&sh.cfull), 1);
+        mbar_init(smem_u32(&sh.cempty), 2); // both MMA issuers release the covariance blocks
+        mbar_init(smem_u32(&sh.done[0]), 1);
+        mbar_init(smem_u32(&sh.done[1]), 1);
+        sh.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    const int hpb = p.tc_hpb, my_hs = p.H / hpb;
+    const int my_h0 = blockIdx.x % my_hs, my_group = blockIdx.x / my_hs;
+    tc_partition(p, gridDim.x / my_hs, prefix, &sh.tiles_lh, &sh.n_tiles, &sh.tpc);
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)), "r"(512) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = sh.tmem_base;
+    const int tiles_lh = sh.tiles_lh, tpc = sh.tpc;
+    const long long g_begin = (long long)my_group * tpc;
+    const long long g_end = (g_begin + tpc < sh.n_tiles) ? g_begin + tpc : sh.n_tiles;
+    const long long g_span = g_end - g_begin;
+    const float c_lin = kLog2e * 0.08838834764831845f; // log2(e) / sqrt(128)
+    const float c_quad = kLog2e * (1.0f / 256.0f);     // log2(e) / (2 * 128)
+
+    if (tiles_lh > 0 && g_begin < g_end) {
+        if (warp == 0) {
+            // ------------------------------------------------------------ TMA producer
+            int kit = 0, seg = 0, issued = 0;
+            bool ok = true;
+            for (long long gv = 0; gv < g_span * hpb && ok;) {
+                const int my_h = my_h0 + (int)(gv / g_span) * my_hs;
+                const long long g = g_begin + gv % g_span;
+                const Segment s = decode_segment(p, prefix, tiles_lh, tpc, g, g_end, my_h);
+                ok = mbar_wait(smem_u32(&sh.cempty), (uint32_t)((seg & 1) ^ 1), abort_flag);
+                if (!ok) break;
+                if (lane == 0) {
+                    mbar_expect_tx(smem_u32(&sh.cfull), (uint32_t)(n_rb * kTileBytes));
+                    const int crow0 = ((((s.l * p.B + s.b) * p.H + s.h) * p.G) + p.ex_g0) * kHeadDim;
+                    for (int rb = 0; rb < n_rb; ++rb)
+                        for (int hf = 0; hf < 2; ++hf)
+                            tma_load_2d(smem_u32(Cs + (size_t)rb * kTileBytes + hf * kHalfBytes), &c_map, smem_u32(&sh.cfull),
+                                        hf * 64, crow0 + rb * kHeadDim);
+                }
+                const int *table = p.block_table + (size_t)s.b * p.bt_stride;
+                const int last_page = (s.T - 1) >> 4;
+                for (int i = 0; i < s.n && ok; ++i, ++kit) {
+                    const int st = kit % NS;
+                    ok = mbar_wait(smem_u32(&sh.kempty[st]), (uint32_t)(((kit / NS) & 1) ^ 1), abort_flag);
+                    if (!ok) break;
+                    if (lane == 0) mbar_expect_tx(smem_u32(&sh.kfull[st]), (uint32_t)kTileBytes);
+                    __syncwarp();
+                    if (lane < 8) {
+                        const int pg = lane;
+                        int pi = (s.tile0 + i) * 8 + pg;
+                        if (pi > last_page) pi = last_page; // tokens past the end are dropped by position
+                        tma_load_5d(smem_u32(Ks + (size_t)st * kTileBytes + pg * 4096), &k_map, smem_u32(&sh.kfull[st]), 0, 0, 2 * s.h, 0,
+                                    s.l * (int)p.num_pages + table[pi]);
+                    }
+                    issued = kit + 1;
+                }
+                gv += s.n;
+                ++seg;
+            }
+            if (!ok) { // drain: wait (bounded) for the copies that were issued and never consumed
+                for (int k = max(0, issued - NS); k < issued; ++k) {
+                    for (uint32_t i = 0; i < kWaitLimit; ++i)
+                        if (mbar_try_wait(smem_u32(&sh.kfull[k % NS]), (uint32_t)((k / NS) & 1))) break;
+                }
+            }
+        } else if (warp == 1 || warp == 3) {
+            // ------------------------------------------------------------ MMA issuers (one per consumer pair)
+            if (lane == 0) {
+                const int wg = warp >> 1;
+                int kit = 0, seg = 0, wsit = 0;
+                bool ok = true;
+                for (long long gv = 0; gv < g_span * hpb && ok;) {
+                    const int my_h = my_h0 + (int)(gv / g_span) * my_hs;
+                    const long long g = g_begin + gv % g_span;
+                    const Segment s = decode_segment(p, prefix, tiles_lh, tpc, g, g_end, my_h);
+                    ok = mbar_wait(smem_u32(&sh.cfull), (uint32_t)(seg & 1), abort_flag);
+                    for (int i = 0; i < s.n && ok; ++i, ++kit) {
+                        if ((kit & 1) != wg) continue;
+                        const int st = kit % NS;
+                        ok = mbar_wait(smem_u32(&sh.kfull[st]), (uint32_t)((kit / NS) & 1), abort_flag);
+                        for (int rb = 0; rb < n_rb && ok; ++rb, ++wsit) {
+                            const int slot = 2 * wg + (wsit & 1);
+                            ok = mbar_wait(smem_u32(&sh.tempty[slot]), (uint32_t)(((wsit >> 1) & 1) ^ 1), abort_flag);
+                            if (!ok) break;
+                            tc_fence_after();
+                            const uint32_t ca = smem_u32(Cs + (size_t)rb * kTileBytes), ka = smem_u32(Ks + (size_t)st * kTileBytes);
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                const unsigned long long dc = smem_desc(ca + (uint32_t)((k >> 2) * kHalfBytes + (k & 3) * 32), 1024);
+                                const unsigned long long dk = smem_desc(ka + (uint32_t)((k >> 2) * 1024 + (k & 3) * 32), 2048);
+                                tc_mma(tmem_base + (uint32_t)(slot * 128), dk, dc, kIdesc, k > 0); // D[t][j] = sum_i K[t][i] C[j][i]
+                            }
+                            tc_commit(smem_u32(&sh.tfull[slot]));
+                        }
+                        if (ok) tc_commit(smem_u32(&sh.kempty[st]));
+                    }
+                    if (ok) tc_commit(smem_u32(&sh.cempty));
+                    gv += s.n;
+                    ++seg;
+                }
+                tc_commit(smem_u32(&sh.done[wg]));
+                for (uint32_t i = 0; i < kWaitLimit; ++i)
+                    if (mbar_try_wait(smem_u32(&sh.done[wg]), 0)) break;
+            }
+            __syncwarp();
+        } else if (warp >= 4) {
+            // ------------------------------------------------------------ consumers
+            const int wgq = (warp - 4) >> 2, pair = wgq & 1, half = wgq >> 1, quad = warp & 3, li = quad * 32 + lane;
+            int kit = 0, wsit = 0, seg = 0, pc0 = 0, pc1 = 0;
+            bool ok = true;
+            for (long long gv = 0; gv < g_span * hpb;) {
+                const int my_h = my_h0 + (int)(gv / g_span) * my_hs;
+                const long long g = g_begin + gv % g_span;
+                const Segment s = decode_segment(p, prefix, tiles_lh, tpc, g, g_end, my_h);
+                const int T = s.T;
+                const int sti = pair * 128 + li; // this thread's place in the statistics (first half only)
+                if (half == 0)
+                    for (int rb = 0; rb < kExHeads; ++rb) sh.stat[rb][sti] = make_float2(-INFINITY, 0.0f);
+                // this unit's means, scaled once; the buffer alternates between segments and the barrier below
+                // keeps the consumers within one segment of each other
+                float *mu = mu_s + (seg & 1) * n_rb * kHeadDim;
+                {
+                    const float *mu_g = p.q_mean + ((size_t)s.uid * p.G + p.ex_g0) * kHeadDim;
+                    for (int i = (warp - 4) * 32 + lane; i < n_rb * kHeadDim; i += kConsumerThreads) mu[i] = mu_g[i] * c_lin;
+                }
+                asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
+                float *lg_out = p.ex_logits + ((size_t)s.uid * p.G + p.ex_g0) * p.T_cap;
+                for (int i = 0; i < s.n && ok; ++i, ++kit) {
+                    if ((kit & 1) != pair) continue;
+                    const int t0 = (s.tile0 + i) * kTileTokens;
+                    const int st = kit % NS;
+                    ok = mbar_wait(smem_u32(&sh.kfull[st]), (uint32_t)((kit / NS) & 1), abort_flag);
+                    if (!ok) break;
+                    // this thread's half of its token's key: eight 16-byte chunks, un-swizzled by the row number
+                    unsigned kw[32];
+                    {
+                        const unsigned char *row = Ks + (size_t)st * kTileBytes + (li >> 3) * 2048 + half * 1024 + (li & 7) * 128;
+#pragma unroll
+                        for (int cch = 0; cch < 8; ++cch) {
+                            const uint4 v = *reinterpret_cast<const uint4 *>(row + ((cch ^ (li & 7)) << 4));
+                            kw[4 * cch] = v.x; kw[4 * cch + 1] = v.y; kw[4 * cch + 2] = v.z; kw[4 * cch + 3] = v.w;
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&sh.kempty[st]));
+                    for (int rb = 0; rb < n_rb && ok; ++rb, ++wsit) {
+                        const int slot = 2 * pair + (wsit & 1);
+                        ok = mbar_wait(smem_u32(&sh.tfull[slot]), (uint32_t)((wsit >> 1) & 1), abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * 128 + half * 64);
+                        // chunks of 8 columns, the load of the next chunk in flight while this one is worked on
+                        uint32_t buf[2][8];
+                        tc_ld8_issue(taddr, buf[0]);
+                        tc_ld8_wait(buf[0]);
+                        const float4 *mu4 = reinterpret_cast<const float4 *>(mu + rb * kHeadDim + half * 64);
+                        unsigned long long aq2 = 0ull, al2 = 0ull; // packed (0.0f, 0.0f)
+#pragma unroll
+                        for (int ch = 0; ch < 8; ++ch) {
+                            uint32_t (&cur)[8] = buf[ch & 1];
+                            if (ch < 7) tc_ld8_issue(taddr + (ch + 1) * 8, buf[(ch + 1) & 1]);
+#pragma unroll
+                            for (int j4 = 0; j4 < 2; ++j4) {
+                                const float4 f = mu4[ch * 2 + j4];
+                                const unsigned w0 = kw[ch * 4 + 2 * j4], w1 = kw[ch * 4 + 2 * j4 + 1];
+                                const unsigned long long k0 = pack_f32x2(bf16_lo(w0), bf16_hi(w0));
+                                const unsigned long long k1 = pack_f32x2(bf16_lo(w1), bf16_hi(w1));
+                                aq2 = fma_f32x2(pack_f32x2(__uint_as_float(cur[4 * j4]), __uint_as_float(cur[4 * j4 + 1])), k0, aq2);
+                                al2 = fma_f32x2(pack_f32x2(f.x, f.y), k0, al2);
+                                aq2 = fma_f32x2(pack_f32x2(__uint_as_float(cur[4 * j4 + 2]), __uint_as_float(cur[4 * j4 + 3])), k1, aq2);
+                                al2 = fma_f32x2(pack_f32x2(f.z, f.w), k1, al2);
+                            }
+                            if (ch < 7) tc_ld8_wait(buf[(ch + 1) & 1]);
+                        }
+                        float val = fmaf(sum_f32x2(aq2), c_quad, sum_f32x2(al2)); // this half's part of the logit, in log2 units
+                        // The two halves of the columns meet here: the second warpgroup leaves its part in shared memory,
+                        // the first adds it.  The buffer belongs to the slot, and the first warpgroup releases the slot only
+                        // after reading it, so the next use of the slot cannot overwrite it early.
+                        const int bit = slot & 1;
+                        float *pa = sh.pacc[pair][bit];
+                        const uint32_t pbar = smem_u32(&sh.pfull[pair][bit]);
+                        if (half == 1) {
+                            pa[li] = val;
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) { mbar_arrive(pbar); mbar_arrive(smem_u32(&sh.tempty[slot])); }
+                        } else {
+                            ok = mbar_wait(pbar, (uint32_t)((bit ? pc1 : pc0) & 1), abort_flag);
+                            if (ok) {
+                                val += pa[li];
+                                const int t = t0 + li;
+                                if (t < T) {
+                                    lg_out[(size_t)rb * p.T_cap + t] = val;
+                                    const float2 mz = sh.stat[rb][sti];
+                                    const float mn = fmaxf(mz.x, val);
+                                    sh.stat[rb][sti] = make_float2(mn, mz.y * ex2(mz.x - mn) + ex2(val - mn));
+                                }
+                                tc_fence_before();
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(smem_u32(&sh.tempty[slot]));
+                            }
+                        }
+                        if (bit) ++pc1; else ++pc0;
+                    }
+                }
+                // fold the first-half warps' statistics in a fixed order and store this block's part of the unit
+                if (half == 0) {
+#pragma unroll
+                    for (int rb = 0; rb < kExHeads; ++rb) {
+                        float mm = sh.stat[rb][sti].x, zz = sh.stat[rb][sti].y;
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) {
+                            const float m2 = __shfl_xor_sync(0xffffffffu, mm, o), z2 = __shfl_xor_sync(0xffffffffu, zz, o);
+                            lse_merge(mm, zz, m2, z2);
+                        }
+                        if (lane == 0) sh.red[pair * 4 + quad][rb] = make_float2(mm, zz);
+                    }
+                }
+                asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
+                if (warp == 4 && lane < n_rb && ok) {
+                    float mm = -INFINITY, zz = 0.0f;
+                    for (int w = 0; w < 8; ++w) lse_merge(mm, zz, sh.red[w][lane].x, sh.red[w][lane].y);
+                    reinterpret_cast<float2 *>(p.part)[((size_t)s.uid * p.n_slices + s.part) * p.G + p.ex_g0 + lane] = make_float2(mm, zz);
+                }
+                asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory"); // the buffer is free again
+                gv += s.n;
+                ++seg;
+            }
+        }
+    }
+    if (*abort_flag && tid == 0) set_status(p.status, AMS_ERR_TIMEOUT, blockIdx.x, 3, 0);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+}
+
+constexpr int kFinThreads = 256; // 16 token rows x 16 lanes of 16 bytes
+
+// score_t = (mean over the group's heads of 2^(l_{r,t} - b_r) + eps) * |v_t|, b_r = M_r + log2 Z_r merged from the
+// parts the blocks of the first kernel left (an unused part is all zero).
+__global__ void __launch_bounds__(kFinThreads) k_expected_final(DevParams p)
+{
+    __shared__ float b_s[16];
+    wait_for_previous_kernel(); // logits and statistics
+    const int uid = blockIdx.y, slice = blockIdx.x;
+    const int h = uid % p.H, b = (uid / p.H) % p.B, l = uid / (p.H * p.B);
+    const int T = p.seq_lens[b];
+    if (T <= p.Tk || T > p.T_cap) return;
+    const int t_begin = slice * p.slice_len;
+    if (t_begin >= T) return;
+    const int t_end = min(T, t_begin + p.slice_len);
+    if (threadIdx.x < p.G) {
+        float mm = -INFINITY, zz = 0.0f;
+        for (int q = 0; q < p.n_slices; ++q) {
+            const float2 v = __ldcg(reinterpret_cast<const float2 *>(p.part) + ((size_t)uid * p.n_slices + q) * p.G + threadIdx.x);
+            if (v.y > 0.0f) lse_merge(mm, zz, v.x, v.y);
+        }
+        b_s[threadIdx.x] = zz > 0.0f ? mm + log2f(zz) : INFINITY;
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 15, r = threadIdx.x >> 4;
+    const int *table = p.block_table + (size_t)b * p.bt_stride;
+    const float *lg = p.ex_logits + (size_t)uid * p.G * p.T_cap;
+    const float my_b = lane < p.G ? b_s[lane] : INFINITY;
+    const float inv_g = 1.0f / (float)p.G;
+    float *g_out = p.scores + (size_t)uid * p.T_cap;
+    constexpr int kU = 4; // tokens per thread and round: their loads are issued together
+    const int n_iter = (t_end - t_begin + 16 * kU - 1) / (16 * kU);
+    for (int it = 0; it < n_iter; ++it) {
+        uint4 v[kU];
+        float e[kU];
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+            const int t = t_begin + (it * kU + u) * 16 + r;
+            v[u] = make_uint4(0, 0, 0, 0);
+            e[u] = -INFINITY;
+            if (t < t_end) {
+                v[u] = ld_stream16(p.v_pages + row_offset(p, l, table[t >> 4], t & 15, h) + lane * 8);
+                if (lane < p.G) e[u] = __ldcs(lg + (size_t)lane * p.T_cap + t);
+            }
+        }
+        float a[2 * kU]; // a[2u]: this lane's part of |v|^2 of token u; a[2u + 1]: its head's attention weight
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+            const unsigned w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+            unsigned long long sq2 = 0ull;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const unsigned long long x2 = pack_f32x2(bf16_lo(w[i]), bf16_hi(w[i]));
+                sq2 = fma_f32x2(x2, x2, sq2);
+            }
+            a[2 * u] = sum_f32x2(sq2);
+            a[2 * u + 1] = tc::ex2(e[u] - my_b); // lanes beyond the group: 2^(-inf) = 0
+        }
+        // sums over the 16 lanes of a token row, all eight values at once: at each step a lane hands half of
+        // its values to its partner and keeps the other half
+#pragma unroll
+        for (int o = 8, n = 2 * kU; o >= 2; o >>= 1, n >>= 1) {
+            const bool up = (lane & o) != 0;
+#pragma unroll
+            for (int i = 0; i < n / 2; ++i) {
+                const float send = up ? a[i] : a[i + n / 2];
+                const float keep = up ? a[i + n / 2] : a[i];
+                a[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+            }
+        }
+        a[0] += __shfl_xor_sync(0xffffffffu, a[0], 1);
+        // lane holds value index 4 * bit3 + 2 * bit2 + bit1: even = |v|^2 of token (index / 2), odd = its weight sum
+        const float other = __shfl_xor_sync(0xffffffffu, a[0], 2);
+        if ((lane & 3) == 0) {
+            const int u = lane >> 2;
+            const int t = t_begin + (it * kU + u) * 16 + r;
+            if (t < t_end) g_out[t] = fmaf(other, inv_g, p.score_eps) * sqrtf(a[0]);
+        }
+    }
+}
+
+} // namespace
+
+bool expected_supported(const DevParams &p) { return p.G >= 1 && p.G <= 16 && p.B <= 1024 && p.H <= 64; }
+
+int launch_score_expected(const DevParams &p_in, LaunchCtx &ctx)
+{
+    DevParams p = p_in;
+    if (!p.q_mean || !p.q_cov || !p.ex_logits) return AMS_ERR_INVALID_ARG;
+    if (!expected_supported(p)) return AMS_ERR_UNSUPPORTED;
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return AMS_ERR_CUDA;
+    CUtensorMap k_map, c_map;
+    int rc = make_k_map(p, enc, &k_map);
+    if (rc == AMS_OK) rc = make_rows_map(p.q_cov, (unsigned long long)p.L * p.B * p.H * p.G * kHeadDim, enc, &c_map);
+    if (rc != AMS_OK) return rc;
+    const int n_sm = sm_count();
+    if (n_sm <= 0) return AMS_ERR_CUDA;
+    const TcGrid tg = tc_grid(p, n_sm);
+    p.tc_hpb = tg.hpb;
+    // unused parts of the statistics must read as empty
+    const size_t U = (size_t)p.L * p.B * p.H;
+    if (cudaMemsetAsync(p.part, 0, U * p.n_slices * p.G * sizeof(float2), ctx.s) != cudaSuccess) return AMS_ERR_CUDA;
+    static SmemGrant grant;
+    for (int g0 = 0; g0 < p.G; g0 += kExHeads) {
+        p.ex_g0 = g0;
+        p.ex_gc = p.G - g0 < kExHeads ? p.G - g0 : kExHeads;
+        // an even ring depth: each stage then belongs to one of the two MMA issuers
+        p.tc_stages = p.ex_gc <= 2 ? 4 : 2;
+        const size_t smem = 1024 + (size_t)(p.ex_gc + p.tc_stages) * kTileBytes + (size_t)2 * p.ex_gc * kHeadDim * 4 + 256;
+        if (!grant_dynamic_smem(k_expected_tc, smem, grant)) return AMS_ERR_CUDA;
+        k_expected_tc<<<tg.grid, kTcThreads, smem, ctx.s>>>(p, k_map, c_map);
+        ctx.mark(kKernScore1);
+    }
+    const dim3 grid(p.n_slices, (unsigned)U);
+    if (launch_after(k_expected_final, grid, dim3(kFinThreads), 0, ctx.s, p) != cudaSuccess) return AMS_ERR_CUDA;
+    ctx.mark(kKernScore2);
+    return cudaGetLastError() == cudaSuccess ? AMS_OK : AMS_ERR_CUDA;
+}
+
+} // namespace ams

@@ -58,6 +58,12 @@ def test_sizes_and_validation_without_gpu():
         for k, v in kw.items():
             setattr(c, k, v)
         assert lib.ams_workspace_bytes(ctypes.byref(c)) == plain + per_token
+    # the expected-attention scorer keeps one logit per query head and token
+    c = binding.config_for(inputs.CONFIGS[0], expected_scorer=1)
+    assert lib.ams_workspace_bytes(ctypes.byref(c)) == plain + per_token * (cfg.n_q_heads // cfg.n_kv_heads)
+    c.expected_scorer = 2
+    assert lib.ams_workspace_bytes(ctypes.byref(c)) == 0
+    assert lib.ams_set_query_stats(None, None, None, ctypes.c_float(0.01)) == binding.AMS_ERR_INVALID_ARG
     assert binding.strerror(binding.AMS_ERR_TIMEOUT) == "bounded device wait expired"
     handle = ctypes.c_void_p()
     rc = lib.ams_init_state(ctypes.byref(cfg), None, None, 0, None, ctypes.byref(handle))
