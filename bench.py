@@ -84,7 +84,7 @@ def config_dict(wl) -> dict:
            else "chosen with --config")
     return {"workload": wl.name, "layers": wl.n_layers, "layers_resident": wl.layers_resident, "q_heads": wl.n_q_heads,
             "kv_heads": wl.n_kv_heads, "batch_per_gpu": wl.batch, "cache_tokens": wl.seq_len_max, "budget": wl.budget,
-            "window": wl.window, "n_segments": wl.n_segments, "scorer": "tova" if wl.scorer_id == 0 else "keydiff",
+            "window": wl.window, "n_segments": wl.n_segments, "scorer": SCORER_NAMES[wl.scorer_id],
             "event": "first event (cache at full length); steady-state events are under per_config",
             "why_this_workload": why}
 
@@ -93,7 +93,7 @@ def algorithmic_bytes(wl, lens) -> tuple[int, int]:
     """(K bytes read once for scoring, kept K/V bytes read + written) per step."""
     units = wl.layers_resident * wl.n_kv_heads
     live = [int(t) for t in lens if int(t) > wl.budget]
-    k_read = units * sum(live) * 256
+    k_read = units * sum(live) * (512 if wl.scorer_id == 3 else 256)   # the expected-attention scorer also reads V (value norms)
     moved = units * len(live) * wl.budget * 2 * 256 * 2
     return k_read, moved
 
@@ -178,6 +178,10 @@ class Bench:
         self.dst = torch.from_numpy(self.dst_np).to(dev)
         self.table0, self.lens0 = self.cache.block_table.clone(), self.cache.seq_lens.clone()
         self.q = self.cache.obs_queries if wl.scorer_id == inputs.SCORER_TOVA else None
+        self.stats = None
+        if wl.scorer_id == inputs.SCORER_EXPECTED:
+            self.stats = inputs.make_query_stats(self.cache)
+            self.comp.set_query_stats(self.stats[0], self.stats[1], 1e-2)
         k_read, moved = algorithmic_bytes(wl, self.lens0.cpu().numpy())
         self.k_read, self.moved = k_read, moved
         # inputs smaller than twice the L2 are flushed out of it between timed steps
@@ -225,12 +229,13 @@ class Bench:
 
     def close(self):
         self.comp.close()
-        for name in ("cache", "comp", "dst", "table0", "lens0", "q", "flush"):
+        for name in ("cache", "comp", "dst", "table0", "lens0", "q", "flush", "stats"):
             setattr(self, name, None)
         gc.collect()
         torch.cuda.empty_cache()
 
 
+SCORER_NAMES = {0: "tova", 1: "keydiff", 2: "external", 3: "expected_attention"}
 SCORE_SLOTS = ("score_phase1", "score_combine", "score_phase2")
 SELECT_SLOTS = ("segment_select", "segments_quotas", "select_compact")
 
@@ -252,6 +257,11 @@ def roofline_of(wl, kern_ms, k_read, moved, lens, peaks, traffic=None):
                     f"quoted for the longest kernel that does")
     if dom == "gather":
         bytes_launch, bound = moved, "hbm"
+    elif wl.scorer_id == 3 and dom == "score_phase1":
+        # K once (the V pass is the other scorer kernel); 2 * 128 * 128 flops per (query head, token) on the tensor pipe
+        bytes_launch, bound = k_read // 2, "tensor"
+    elif wl.scorer_id == 3:
+        bytes_launch, bound = k_read // 2, "hbm"
     else:
         bytes_launch = k_read
         # wide query blocks: two passes with one exponential and one multiply-add per (row, token, d) each; the
@@ -263,6 +273,15 @@ def roofline_of(wl, kern_ms, k_read, moved, lens, peaks, traffic=None):
     if bound == "hbm":
         out.update(achieved=hbm_achieved, peak=peaks["hbm_gbs"], unit="GB/s", frac=hbm_achieved / peaks["hbm_gbs"])
         note.append("achieved = algorithmic bytes of the launch / mean CUDA-event duration of that kernel; frac is of the measured copy bandwidth")
+    elif bound == "tensor":
+        token_heads = wl.layers_resident * wl.n_kv_heads * sum(int(t) for t in lens if int(t) > wl.budget)
+        flops = token_heads * wl.group * 2 * 128 * 128
+        achieved = flops / (ms * 1e-3) / 1e12
+        out.update(achieved=achieved, peak=peaks["bf16_tflops"], unit="TFLOP/s", frac=achieved / peaks["bf16_tflops"],
+                   operations_per_launch=flops,
+                   also={"hbm_gbs": hbm_achieved, "hbm_frac": hbm_achieved / peaks["hbm_gbs"]})
+        note.append("one 128 x 128 matrix-vector product per (query head, token) on the tensor pipe (K tile x covariance), bf16 in, "
+                    "fp32 accumulate; frac is of the measured cuBLAS bf16 rate (burst); the K stream of the same launch is under 'also'")
     else:
         token_heads = wl.layers_resident * wl.n_kv_heads * sum(int(t) for t in lens if int(t) > wl.budget)
         exps = token_heads * rows
@@ -340,7 +359,7 @@ def measure_config(cfg_id, dev, steps, warmup, peaks, layers=0, with_steady=True
         "workload": wl.name, "layers_resident": wl.layers_resident, "layers_total": wl.n_layers, "batch": wl.batch,
         "kv_heads": wl.n_kv_heads, "query_rows_per_kv_head": wl.group * max(wl.window, 1),
         "cache_tokens": [int(lens.min()), int(lens.max())], "budget": wl.budget, "n_segments": wl.n_segments,
-        "scorer": "tova" if wl.scorer_id == 0 else "keydiff", "steps": steps,
+        "scorer": SCORER_NAMES[wl.scorer_id], "steps": steps,
         "ms_per_step": ms, "ms_per_step_min": float(np.min(per_step)), "steps_per_s": 1e3 / ms,
         "algorithmic_bytes_per_step": total, "effective_hbm_gbs": total / (ms * 1e-3) / 1e9,
         "effective_hbm_frac_of_8tbs": total / (ms * 1e-3) / 8e12,
@@ -367,12 +386,14 @@ def e2e_loop(b: Bench, n_e2e):
     host_q = q.cpu().pin_memory() if q is not None else None
     host_table, host_lens, host_dst = b.table0.cpu().pin_memory(), b.lens0.cpu().pin_memory(), dst.cpu().pin_memory()
     out_table, out_lens = torch.empty_like(host_table).pin_memory(), torch.empty_like(host_lens).pin_memory()
-    h2d = sum(t.numel() * t.element_size() for t in (host_q, host_table, host_lens, host_dst) if t is not None)
+    host_stats = [t.cpu().pin_memory() for t in b.stats] if b.stats is not None else None   # query statistics of this event
+    h2d = sum(t.numel() * t.element_size() for t in (host_q, host_table, host_lens, host_dst, *(host_stats or [])) if t is not None)
     d2h = out_table.numel() * 4 + out_lens.numel() * 4 + 16
     NB = 3
     sets = [(q, cache.block_table, cache.seq_lens, dst)] + [
         (None if q is None else torch.empty_like(q), torch.empty_like(cache.block_table), torch.empty_like(cache.seq_lens),
          torch.empty_like(dst)) for _ in range(NB - 1)]
+    stat_sets = None if b.stats is None else [b.stats] + [tuple(torch.empty_like(t) for t in b.stats) for _ in range(NB - 1)]
     copy_stream, read_stream = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
     uploaded = [torch.cuda.Event() for _ in range(NB)]
     computed = [torch.cuda.Event() for _ in range(NB)]
@@ -388,6 +409,9 @@ def e2e_loop(b: Bench, n_e2e):
             ti.copy_(host_table, non_blocking=True)
             li.copy_(host_lens, non_blocking=True)
             di.copy_(host_dst, non_blocking=True)
+            if stat_sets is not None:
+                for dev_t, host_t in zip(stat_sets[i % NB], host_stats):
+                    dev_t.copy_(host_t, non_blocking=True)
             uploaded[i % NB].record(copy_stream)
 
     def check(i):                           # results of step i: wait for their read-back and look at them
@@ -401,6 +425,8 @@ def e2e_loop(b: Bench, n_e2e):
         upload(i + 1)                       # overlaps the kernels of steps i - 1 and i
         stream.wait_event(uploaded[i % NB])
         comp.ema_state.zero_()
+        if stat_sets is not None:
+            comp.set_query_stats(stat_sets[i % NB][0], stat_sets[i % NB][1], 1e-2)
         comp.compress(cache.k_pages, cache.v_pages, ti, li, qi, wl.budget, wl.n_segments, wl.scorer_id, di)
         computed[i % NB].record(stream)
         with torch.cuda.stream(read_stream):  # block table and lengths of this step back to pinned host memory
@@ -527,6 +553,11 @@ def run_ours(args, rank, world, local_rank):
             bb.close()
             per[f"cfg{cid}"] = entry
         out["per_config"] = per
+        # beyond the five benchmark configurations: the expected-attention scorer on the geometry of configuration 1
+        bb, entry, _ = measure_config(5, dev, min(args.steps, 10), 3, peaks)
+        bb.close()
+        entry["note"] = "extension, not one of the five benchmark configurations: expected-attention scorer (tensor-core kernel over K, then a pass over V)"
+        out["extensions"] = {"cfg5": entry}
     elif steady_head:
         out["steady_state"] = steady_head
     if world > 1:
@@ -547,6 +578,10 @@ def _oracle_sample(wl, cache, dst_np, table0, lens0, units):
     v = inputs.as_u16(cache.v_pages.index_select(0, idx))
     q = inputs.as_u16(cache.obs_queries.index_select(0, idx)) if cache.obs_queries is not None else None
     table, lens = table0.cpu().numpy(), lens0.cpu().numpy()
+    stats = {}
+    if wl.scorer_id == inputs.SCORER_EXPECTED:
+        mean, cov = inputs.make_query_stats(cache)
+        stats = dict(q_mean=mean.index_select(0, idx).cpu().numpy(), q_cov=inputs.as_u16(cov.index_select(0, idx)), score_eps=1e-2)
     prm = oracle.Params(wl.n_segments, wl.l_min, wl.l_max, wl.q_min, wl.n_sink, wl.n_last, wl.ema_lambda, wl.ema_beta, wl.eps)
     local_units = [(remap[l], b, h) for (l, b, h) in units]
     oracle.lib()
@@ -554,7 +589,7 @@ def _oracle_sample(wl, cache, dst_np, table0, lens0, units):
     def run(threads):
         credit = np.zeros((len(layers), wl.batch, wl.n_kv_heads, wl.max_seq_len), np.float32)
         oracle.compress(k, v, table.copy(), lens.copy(), q, credit, wl.budget, prm, wl.scorer_id, dst_np,
-                        n_q_heads=wl.n_q_heads, units=local_units, threads=threads)
+                        n_q_heads=wl.n_q_heads, units=local_units, threads=threads, **stats)
     return run
 
 

@@ -7,11 +7,12 @@
 // k_expected_tc reads K once: a 128-token tile is the A operand (tokens on the TMEM lanes) and the
 // group's covariance matrices, resident in shared memory, are the B operands, so that one
 // tcgen05.mma chain per head leaves (Sigma_r k_t) of token t in the 128 columns of TMEM lane t.  The
-// thread that owns the lane dots them with k_t (read from the same shared-memory tile) and with mu_r,
-// stores the logit and keeps a running (max, sum of 2^x) per head.  The block shape and the pipeline are those of
-// the window scorer: warp 0 feeds K tiles by TMA, warps 1 and 3 issue the MMAs for the two consumer
-// pairs, warps 4-19 are four consumer warpgroups (two per tile, each taking 64 of a head's 128
-// columns).  k_expected_final then streams V and the stored logits (16 bytes per token and head
+// thread that owns the lane dots them with k_t (read from the same shared-memory tile); the mean term
+// mu_r . k_t of the tile comes from one more warp (mma.sync on the same tile); the logit is stored and a
+// running (max, sum of 2^x) kept per head.  The block shape and the pipeline are those of
+// the window scorer: warp 0 feeds K tiles by TMA, warp 2 computes the mean terms, warps 1 and 3 issue the MMAs for the two
+// pairs of accumulator slots, warps 4-19 are four consumer warpgroups (each taking 32 of a head's 128
+// columns of every tile).  k_expected_final then streams V and the stored logits (16 bytes per token and head
 // group of four) and writes the scores.  Every wait is bounded; on expiry the block reports
 // AMS_ERR_TIMEOUT, drains its copies, frees its TMEM and returns.
 #include <cuda.h>
@@ -31,10 +32,12 @@ constexpr int kExHeads = 4; // query heads per launch: 4 x 128 accumulator colum
 struct ExShared {
     unsigned long long kfull[kMaxStages], kempty[kMaxStages], tfull[kSlots], tempty[kSlots];
     unsigned long long cfull, cempty, done[2];
-    unsigned long long pfull[2][2];  // the second half's part of a logit is in pacc[pair][slot bit]
-    float pacc[2][2][128];
-    float2 red[8][kExHeads];         // per first-half consumer warp and head: (max, sum of 2^(x - max))
-    float2 stat[kExHeads][256];      // running (max, sum) of every first-half consumer thread, per head
+    unsigned long long pfull[kSlots]; // warpgroups 1-3 have left their parts of a logit in pacc[slot]
+    float pacc[kSlots][3][128];
+    float2 red[4][kExHeads];          // per warp of warpgroup 0 and head: (max, sum of 2^(x - max))
+    float2 stat[kExHeads][128];       // running (max, sum) of every thread of warpgroup 0, per head
+    unsigned long long linfull[2], linempty[2];
+    float lin[2][128][kExHeads];      // mean term of the logits of a tile's tokens, per head (log2 units), two tiles deep
     uint32_t tmem_base;
     int abort_flag;
     int tiles_lh, tpc;
@@ -52,16 +55,19 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_expected_tc(DevParams p, cons
     unsigned char *base = reinterpret_cast<unsigned char *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     unsigned char *Cs = base;                                   // [n_rb][2 halves][128 rows][128 B]
     unsigned char *Ks = Cs + (size_t)n_rb * kTileBytes;         // [NS][8-row group][2 halves][8 rows][128 B]
-    float *mu_s = reinterpret_cast<float *>(Ks + (size_t)NS * kTileBytes); // [2][n_rb][128], scaled
     volatile int *abort_flag = &sh.abort_flag;
 
     if (tid == 0) {
         for (int i = 0; i < kMaxStages; ++i) {
             mbar_init(smem_u32(&sh.kfull[i]), 1);
-            mbar_init(smem_u32(&sh.kempty[i]), 9); // the issuer's commit and the eight consumer warps that read the rows
+            mbar_init(smem_u32(&sh.kempty[i]), 19); // both issuers' commits, the mean-term warp and the sixteen consumer warps
         }
-        for (int i = 0; i < kSlots; ++i) { mbar_init(smem_u32(&sh.tfull[i]), 1); mbar_init(smem_u32(&sh.tempty[i]), 8); }
-        for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&sh.pfull[i >> 1][i & 1]), 4);
+        for (int i = 0; i < kSlots; ++i) {
+            mbar_init(smem_u32(&sh.tfull[i]), 1);
+            mbar_init(smem_u32(&sh.tempty[i]), 16);
+            mbar_init(smem_u32(&sh.pfull[i]), 12);
+        }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&sh.linfull[i]), 1); mbar_init(smem_u32(&sh.linempty[i]), 4); }
         mbar_init(smem_u32(&sh.cfull), 1);
         mbar_init(smem_u32(&sh.cempty), 2); // both MMA issuers release the covariance blocks
         mbar_init(smem_u32(&sh.done[0]), 1);
@@ -134,10 +140,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_expected_tc(DevParams p, cons
                 }
             }
         } else if (warp == 1 || warp == 3) {
-            // ------------------------------------------------------------ MMA issuers (one per consumer pair)
+            // ------------------------------------------------------------ MMA issuers (two heads of every tile each)
             if (lane == 0) {
                 const int wg = warp >> 1;
-                int kit = 0, seg = 0, wsit = 0;
+                int kit = 0, seg = 0;
                 bool ok = true;
                 for (long long gv = 0; gv < g_span * hpb && ok;) {
                     const int my_h = my_h0 + (int)(gv / g_span) * my_hs;
@@ -145,12 +151,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_expected_tc(DevParams p, cons
                     const Segment s = decode_segment(p, prefix, tiles_lh, tpc, g, g_end, my_h);
                     ok = mbar_wait(smem_u32(&sh.cfull), (uint32_t)(seg & 1), abort_flag);
                     for (int i = 0; i < s.n && ok; ++i, ++kit) {
-                        if ((kit & 1) != wg) continue;
                         const int st = kit % NS;
                         ok = mbar_wait(smem_u32(&sh.kfull[st]), (uint32_t)((kit / NS) & 1), abort_flag);
-                        for (int rb = 0; rb < n_rb && ok; ++rb, ++wsit) {
-                            const int slot = 2 * wg + (wsit & 1);
-                            ok = mbar_wait(smem_u32(&sh.tempty[slot]), (uint32_t)(((wsit >> 1) & 1) ^ 1), abort_flag);
+                        // Head rb of every tile goes to accumulator slot rb; this issuer fills slots 2 wg and 2 wg + 1, so
+                        // it sees every phase of their barriers in order (a parity wait must not skip a phase), and the
+                        // tensor pipe may run a whole tile ahead of the consumers.
+                        for (int rb = 2 * wg; rb < n_rb && rb < 2 * wg + 2 && ok; ++rb) {
+                            const int slot = rb;
+                            ok = mbar_wait(smem_u32(&sh.tempty[slot]), (uint32_t)((kit & 1) ^ 1), abort_flag);
                             if (!ok) break;
                             tc_fence_after();
                             const uint32_t ca = smem_u32(Cs + (size_t)rb * kTileBytes), ka = smem_u32(Ks + (size_t)st * kTileBytes);
@@ -173,123 +181,172 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_expected_tc(DevParams p, cons
                     if (mbar_try_wait(smem_u32(&sh.done[wg]), 0)) break;
             }
             __syncwarp();
+        } else if (warp == 2) {
+            // ------------------------------------------------------------ mean-term warp
+            // mu_r . k_t for the tile's 128 tokens and the launch's heads with mma.sync (m16n8k16, fp32 accumulate):
+            // A = 16 token rows of the K tile (ldmatrix from the swizzled tile), B = eight columns, two per head:
+            // mu_r rounded to bf16 and the bf16 of what the rounding lost, so that their sum carries mu_r to 2^-17.
+            int kit = 0;
+            bool ok = true;
+            for (long long gv = 0; gv < g_span * hpb && ok;) {
+                const int my_h = my_h0 + (int)(gv / g_span) * my_hs;
+                const long long g = g_begin + gv % g_span;
+                const Segment s = decode_segment(p, prefix, tiles_lh, tpc, g, g_end, my_h);
+                unsigned breg[8][2];
+                {
+                    const int head = lane >> 3, lost = (lane >> 2) & 1; // column n = lane / 4 = 2 * head + lost
+                    const float *mu_g = p.q_mean + ((size_t)s.uid * p.G + p.ex_g0 + head) * kHeadDim;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)
+#pragma unroll
+                        for (int hb = 0; hb < 2; ++hb) {
+                            const int k0 = ks * 16 + hb * 8 + (lane & 3) * 2;
+                            const float x0 = head < n_rb ? mu_g[k0] : 0.0f, x1 = head < n_rb ? mu_g[k0 + 1] : 0.0f;
+                            __nv_bfloat16 h0 = __float2bfloat16_rn(x0), h1 = __float2bfloat16_rn(x1);
+                            if (lost) {
+                                h0 = __float2bfloat16_rn(x0 - __bfloat162float(h0));
+                                h1 = __float2bfloat16_rn(x1 - __bfloat162float(h1));
+                            }
+                            breg[ks][hb] = (unsigned)__bfloat16_as_ushort(h0) | ((unsigned)__bfloat16_as_ushort(h1) << 16);
+                        }
+                }
+                for (int i = 0; i < s.n && ok; ++i, ++kit) {
+                    const int st = kit % NS, lb = kit & 1;
+                    ok = mbar_wait(smem_u32(&sh.kfull[st]), (uint32_t)((kit / NS) & 1), abort_flag);
+                    if (ok) ok = mbar_wait(smem_u32(&sh.linempty[lb]), (uint32_t)(((kit >> 1) & 1) ^ 1), abort_flag);
+                    ok = __all_sync(0xffffffffu, ok) != 0; // (also brings the lanes back together before ldmatrix)
+                    if (!ok) break;
+                    const uint32_t ka = smem_u32(Ks + (size_t)st * kTileBytes);
+#pragma unroll 2
+                    for (int mb = 0; mb < 8; ++mb) {
+                        float c0 = 0.0f, c1 = 0.0f, c2 = 0.0f, c3 = 0.0f;
+                        const int row = mb * 16 + (lane & 15);
+                        const uint32_t rbase = ka + (uint32_t)((row >> 3) * 2048 + (row & 7) * 128);
+#pragma unroll
+                        for (int ks = 0; ks < 8; ++ks) {
+                            const int c16 = ks * 2 + (lane >> 4); // 16-byte chunk of the row: dims [8 c16, 8 c16 + 8)
+                            const uint32_t addr = rbase + (uint32_t)((c16 >> 3) * 1024 + (((c16 & 7) ^ (row & 7)) << 4));
+                            unsigned a0, a1, a2, a3;
+                            asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                                         : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3) : "r"(addr));
+                            asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                                         : "+f"(c0), "+f"(c1), "+f"(c2), "+f"(c3)
+                                         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(breg[ks][0]), "r"(breg[ks][1]));
+                        }
+                        // this lane holds, for rows lane / 4 and lane / 4 + 8 of the block, both columns of head lane % 4
+                        sh.lin[lb][mb * 16 + (lane >> 2)][lane & 3] = (c0 + c1) * c_lin;
+                        sh.lin[lb][mb * 16 + (lane >> 2) + 8][lane & 3] = (c2 + c3) * c_lin;
+                    }
+                    __syncwarp();
+                    if (lane == 0) { mbar_arrive(smem_u32(&sh.linfull[lb])); mbar_arrive(smem_u32(&sh.kempty[st])); }
+                }
+                gv += s.n;
+            }
         } else if (warp >= 4) {
             // ------------------------------------------------------------ consumers
-            const int wgq = (warp - 4) >> 2, pair = wgq & 1, half = wgq >> 1, quad = warp & 3, li = quad * 32 + lane;
-            int kit = 0, wsit = 0, seg = 0, pc0 = 0, pc1 = 0;
+            // Four warpgroups work on every tile together: thread li of warpgroup q owns TMEM lane li (token
+            // t0 + li) and columns [32 q, 32 q + 32) of each head's accumulator.  Its 32 key elements are widened
+            // to fp32 once per tile and serve all heads.  Head rb of a tile is in accumulator slot rb.
+            const int q4 = (warp - 4) >> 2, quad = warp & 3, li = quad * 32 + lane;
+            int kit = 0, seg = 0;
             bool ok = true;
             for (long long gv = 0; gv < g_span * hpb;) {
                 const int my_h = my_h0 + (int)(gv / g_span) * my_hs;
                 const long long g = g_begin + gv % g_span;
                 const Segment s = decode_segment(p, prefix, tiles_lh, tpc, g, g_end, my_h);
                 const int T = s.T;
-                const int sti = pair * 128 + li; // this thread's place in the statistics (first half only)
-                if (half == 0)
-                    for (int rb = 0; rb < kExHeads; ++rb) sh.stat[rb][sti] = make_float2(-INFINITY, 0.0f);
-                // this unit's means, scaled once; the buffer alternates between segments and the barrier below
-                // keeps the consumers within one segment of each other
-                float *mu = mu_s + (seg & 1) * n_rb * kHeadDim;
-                {
-                    const float *mu_g = p.q_mean + ((size_t)s.uid * p.G + p.ex_g0) * kHeadDim;
-                    for (int i = (warp - 4) * 32 + lane; i < n_rb * kHeadDim; i += kConsumerThreads) mu[i] = mu_g[i] * c_lin;
-                }
+                if (q4 == 0)
+                    for (int rb = 0; rb < kExHeads; ++rb) sh.stat[rb][li] = make_float2(-INFINITY, 0.0f);
                 asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
                 float *lg_out = p.ex_logits + ((size_t)s.uid * p.G + p.ex_g0) * p.T_cap;
                 for (int i = 0; i < s.n && ok; ++i, ++kit) {
-                    if ((kit & 1) != pair) continue;
                     const int t0 = (s.tile0 + i) * kTileTokens;
                     const int st = kit % NS;
                     ok = mbar_wait(smem_u32(&sh.kfull[st]), (uint32_t)((kit / NS) & 1), abort_flag);
                     if (!ok) break;
-                    // this thread's half of its token's key: eight 16-byte chunks, un-swizzled by the row number
-                    unsigned kw[32];
+                    // this thread's quarter of its token's key: four 16-byte chunks, un-swizzled by the row number
+                    unsigned long long kf[16];
                     {
-                        const unsigned char *row = Ks + (size_t)st * kTileBytes + (li >> 3) * 2048 + half * 1024 + (li & 7) * 128;
+                        const unsigned char *row = Ks + (size_t)st * kTileBytes + (li >> 3) * 2048 + (q4 >> 1) * 1024 + (li & 7) * 128;
 #pragma unroll
-                        for (int cch = 0; cch < 8; ++cch) {
-                            const uint4 v = *reinterpret_cast<const uint4 *>(row + ((cch ^ (li & 7)) << 4));
-                            kw[4 * cch] = v.x; kw[4 * cch + 1] = v.y; kw[4 * cch + 2] = v.z; kw[4 * cch + 3] = v.w;
+                        for (int cch = 0; cch < 4; ++cch) {
+                            const uint4 v = *reinterpret_cast<const uint4 *>(row + ((((q4 & 1) * 4 + cch) ^ (li & 7)) << 4));
+                            kf[4 * cch] = pack_f32x2(bf16_lo(v.x), bf16_hi(v.x));
+                            kf[4 * cch + 1] = pack_f32x2(bf16_lo(v.y), bf16_hi(v.y));
+                            kf[4 * cch + 2] = pack_f32x2(bf16_lo(v.z), bf16_hi(v.z));
+                            kf[4 * cch + 3] = pack_f32x2(bf16_lo(v.w), bf16_hi(v.w));
                         }
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&sh.kempty[st]));
-                    for (int rb = 0; rb < n_rb && ok; ++rb, ++wsit) {
-                        const int slot = 2 * pair + (wsit & 1);
-                        ok = mbar_wait(smem_u32(&sh.tfull[slot]), (uint32_t)((wsit >> 1) & 1), abort_flag);
+                    const int lb = kit & 1;
+                    if (q4 == 0) { // the mean terms of this tile (warp 2)
+                        ok = mbar_wait(smem_u32(&sh.linfull[lb]), (uint32_t)((kit >> 1) & 1), abort_flag);
+                        if (!ok) break;
+                    }
+                    for (int rb = 0; rb < n_rb && ok; ++rb) {
+                        const int slot = rb;
+                        const uint32_t use_parity = (uint32_t)(kit & 1);
+                        ok = mbar_wait(smem_u32(&sh.tfull[slot]), use_parity, abort_flag);
                         if (!ok) break;
                         tc_fence_after();
-                        const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * 128 + half * 64);
-                        // chunks of 8 columns, the load of the next chunk in flight while this one is worked on
-                        uint32_t buf[2][8];
-                        tc_ld8_issue(taddr, buf[0]);
-                        tc_ld8_wait(buf[0]);
-                        const float4 *mu4 = reinterpret_cast<const float4 *>(mu + rb * kHeadDim + half * 64);
-                        unsigned long long aq2 = 0ull, al2 = 0ull; // packed (0.0f, 0.0f)
+                        const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * 128 + q4 * 32);
+                        uint32_t d[32];
+                        tc_ld32_issue(taddr, d);
+                        tc_ld_wait(d);
+                        unsigned long long aq2 = 0ull;
 #pragma unroll
-                        for (int ch = 0; ch < 8; ++ch) {
-                            uint32_t (&cur)[8] = buf[ch & 1];
-                            if (ch < 7) tc_ld8_issue(taddr + (ch + 1) * 8, buf[(ch + 1) & 1]);
-#pragma unroll
-                            for (int j4 = 0; j4 < 2; ++j4) {
-                                const float4 f = mu4[ch * 2 + j4];
-                                const unsigned w0 = kw[ch * 4 + 2 * j4], w1 = kw[ch * 4 + 2 * j4 + 1];
-                                const unsigned long long k0 = pack_f32x2(bf16_lo(w0), bf16_hi(w0));
-                                const unsigned long long k1 = pack_f32x2(bf16_lo(w1), bf16_hi(w1));
-                                aq2 = fma_f32x2(pack_f32x2(__uint_as_float(cur[4 * j4]), __uint_as_float(cur[4 * j4 + 1])), k0, aq2);
-                                al2 = fma_f32x2(pack_f32x2(f.x, f.y), k0, al2);
-                                aq2 = fma_f32x2(pack_f32x2(__uint_as_float(cur[4 * j4 + 2]), __uint_as_float(cur[4 * j4 + 3])), k1, aq2);
-                                al2 = fma_f32x2(pack_f32x2(f.z, f.w), k1, al2);
-                            }
-                            if (ch < 7) tc_ld8_wait(buf[(ch + 1) & 1]);
-                        }
-                        float val = fmaf(sum_f32x2(aq2), c_quad, sum_f32x2(al2)); // this half's part of the logit, in log2 units
-                        // The two halves of the columns meet here: the second warpgroup leaves its part in shared memory,
-                        // the first adds it.  The buffer belongs to the slot, and the first warpgroup releases the slot only
+                        for (int j = 0; j < 16; ++j)
+                            aq2 = fma_f32x2(pack_f32x2(__uint_as_float(d[2 * j]), __uint_as_float(d[2 * j + 1])), kf[j], aq2);
+                        float val = sum_f32x2(aq2) * c_quad; // this quarter's part of the quadratic term, in log2 units
+                        // The four quarters of the columns meet here: warpgroups 1-3 leave their parts in shared memory,
+                        // warpgroup 0 adds them.  The buffer belongs to the slot, and warpgroup 0 releases the slot only
                         // after reading it, so the next use of the slot cannot overwrite it early.
-                        const int bit = slot & 1;
-                        float *pa = sh.pacc[pair][bit];
-                        const uint32_t pbar = smem_u32(&sh.pfull[pair][bit]);
-                        if (half == 1) {
-                            pa[li] = val;
+                        const uint32_t pbar = smem_u32(&sh.pfull[slot]);
+                        if (q4 != 0) {
+                            sh.pacc[slot][q4 - 1][li] = val;
                             tc_fence_before();
                             __syncwarp();
                             if (lane == 0) { mbar_arrive(pbar); mbar_arrive(smem_u32(&sh.tempty[slot])); }
                         } else {
-                            ok = mbar_wait(pbar, (uint32_t)((bit ? pc1 : pc0) & 1), abort_flag);
+                            ok = mbar_wait(pbar, use_parity, abort_flag);
                             if (ok) {
-                                val += pa[li];
+                                val += (sh.pacc[slot][0][li] + sh.pacc[slot][1][li]) + (sh.pacc[slot][2][li] + sh.lin[lb][li][rb]);
                                 const int t = t0 + li;
                                 if (t < T) {
                                     lg_out[(size_t)rb * p.T_cap + t] = val;
-                                    const float2 mz = sh.stat[rb][sti];
+                                    const float2 mz = sh.stat[rb][li];
                                     const float mn = fmaxf(mz.x, val);
-                                    sh.stat[rb][sti] = make_float2(mn, mz.y * ex2(mz.x - mn) + ex2(val - mn));
+                                    sh.stat[rb][li] = make_float2(mn, mz.y * ex2(mz.x - mn) + ex2(val - mn));
                                 }
                                 tc_fence_before();
                                 __syncwarp();
                                 if (lane == 0) mbar_arrive(smem_u32(&sh.tempty[slot]));
                             }
                         }
-                        if (bit) ++pc1; else ++pc0;
+                    }
+                    if (q4 == 0 && ok) { // the mean-term buffer may be refilled
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&sh.linempty[lb]));
                     }
                 }
-                // fold the first-half warps' statistics in a fixed order and store this block's part of the unit
-                if (half == 0) {
+                // fold warpgroup 0's statistics in a fixed order and store this block's part of the unit
+                if (q4 == 0) {
 #pragma unroll
                     for (int rb = 0; rb < kExHeads; ++rb) {
-                        float mm = sh.stat[rb][sti].x, zz = sh.stat[rb][sti].y;
+                        float mm = sh.stat[rb][li].x, zz = sh.stat[rb][li].y;
 #pragma unroll
                         for (int o = 16; o > 0; o >>= 1) {
                             const float m2 = __shfl_xor_sync(0xffffffffu, mm, o), z2 = __shfl_xor_sync(0xffffffffu, zz, o);
                             lse_merge(mm, zz, m2, z2);
                         }
-                        if (lane == 0) sh.red[pair * 4 + quad][rb] = make_float2(mm, zz);
+                        if (lane == 0) sh.red[quad][rb] = make_float2(mm, zz);
                     }
                 }
                 asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
                 if (warp == 4 && lane < n_rb && ok) {
                     float mm = -INFINITY, zz = 0.0f;
-                    for (int w = 0; w < 8; ++w) lse_merge(mm, zz, sh.red[w][lane].x, sh.red[w][lane].y);
+                    for (int w = 0; w < 4; ++w) lse_merge(mm, zz, sh.red[w][lane].x, sh.red[w][lane].y);
                     reinterpret_cast<float2 *>(p.part)[((size_t)s.uid * p.n_slices + s.part) * p.G + p.ex_g0 + lane] = make_float2(mm, zz);
                 }
                 asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory"); // the buffer is free again
@@ -415,7 +472,7 @@ int launch_score_expected(const DevParams &p_in, LaunchCtx &ctx)
         p.ex_gc = p.G - g0 < kExHeads ? p.G - g0 : kExHeads;
         // an even ring depth: each stage then belongs to one of the two MMA issuers
         p.tc_stages = p.ex_gc <= 2 ? 4 : 2;
-        const size_t smem = 1024 + (size_t)(p.ex_gc + p.tc_stages) * kTileBytes + (size_t)2 * p.ex_gc * kHeadDim * 4 + 256;
+        const size_t smem = 1024 + (size_t)(p.ex_gc + p.tc_stages) * kTileBytes + 256;
         if (!grant_dynamic_smem(k_expected_tc, smem, grant)) return AMS_ERR_CUDA;
         k_expected_tc<<<tg.grid, kTcThreads, smem, ctx.s>>>(p, k_map, c_map);
         ctx.mark(kKernScore1);

@@ -97,6 +97,8 @@ CONFIGS = {
                 SCORER_KEYDIFF, n_segments=16, l_max=4096, ema_beta=1.0, resident_layers=4),
     4: Workload("cfg4_llama70b_L80_T131072_k8192_w64", 4, 80, 64, 8, 1, 131072, 131072, 8192, 64,
                 SCORER_TOVA, n_segments=32, l_max=8192, steps=8, append_per_step=512),
+    # not one of the five benchmark configurations: the geometry of configuration 1 with the expected-attention scorer
+    5: Workload("cfg5_llama8b_L32_T16384_k2048_expected", 5, 32, 32, 8, 1, 16384, 16384, 2048, 0, SCORER_EXPECTED),
 }
 
 
