@@ -32,10 +32,9 @@ constexpr int kExHeads = 4; // query heads per launch: 4 x 128 accumulator colum
 struct ExShared {
     unsigned long long kfull[kMaxStages], kempty[kMaxStages], tfull[kSlots], tempty[kSlots];
     unsigned long long cfull, cempty, done[2];
-    unsigned long long pfull[kSlots]; // warpgroups 1-3 have left their parts of a logit in pacc[slot]
-    float pacc[kSlots][3][128];
-    float2 red[4][kExHeads];          // per warp of warpgroup 0 and head: (max, sum of 2^(x - max))
-    float2 stat[kExHeads][128];       // running (max, sum) of every thread of warpgroup 0, per head
+    float pacc[kSlots][3][128];       // the parts of a logit that the three other warpgroups computed, per slot
+    float2 red[4][kExHeads];          // per warp of warpgroup rb: (max, sum of 2^(x - max)) of head rb
+    float2 stat[kExHeads][128];       // running (max, sum) of head rb in every thread of warpgroup rb
     unsigned long long linfull[2], linempty[2];
     float lin[2][128][kExHeads];      // mean term of the logits of a tile's tokens, per head (log2 units), two tiles deep
     uint32_t tmem_base;
@@ -65,9 +64,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_expected_tc(DevParams p, cons
         for (int i = 0; i < kSlots; ++i) {
             mbar_init(smem_u32(&sh.tfull[i]), 1);
             mbar_init(smem_u32(&sh.tempty[i]), 16);
-            mbar_init(smem_u32(&sh.pfull[i]), 12);
         }
-        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&sh.linfull[i]), 1); mbar_init(smem_u32(&sh.linempty[i]), 4); }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&sh.linfull[i]), 1); mbar_init(smem_u32(&sh.linempty[i]), (uint32_t)(4 * n_rb)); }
         mbar_init(smem_u32(&sh.cfull), 1);
         mbar_init(smem_u32(&sh.cempty), 2); // both MMA issuers release the covariance blocks
         mbar_init(smem_u32(&sh.done[0]), 1);
@@ -217,25 +215,31 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_expected_tc(DevParams p, cons
                     ok = __all_sync(0xffffffffu, ok) != 0; // (also brings the lanes back together before ldmatrix)
                     if (!ok) break;
                     const uint32_t ka = smem_u32(Ks + (size_t)st * kTileBytes);
-#pragma unroll 2
-                    for (int mb = 0; mb < 8; ++mb) {
-                        float c0 = 0.0f, c1 = 0.0f, c2 = 0.0f, c3 = 0.0f;
-                        const int row = mb * 16 + (lane & 15);
-                        const uint32_t rbase = ka + (uint32_t)((row >> 3) * 2048 + (row & 7) * 128);
+                    // eight blocks of 16 tokens, their accumulators independent of one another
+                    float c[8][4];
 #pragma unroll
-                        for (int ks = 0; ks < 8; ++ks) {
-                            const int c16 = ks * 2 + (lane >> 4); // 16-byte chunk of the row: dims [8 c16, 8 c16 + 8)
-                            const uint32_t addr = rbase + (uint32_t)((c16 >> 3) * 1024 + (((c16 & 7) ^ (row & 7)) << 4));
+                    for (int mb = 0; mb < 8; ++mb) c[mb][0] = c[mb][1] = c[mb][2] = c[mb][3] = 0.0f;
+                    const int row = lane & 15; // row of the block whose address this lane supplies to ldmatrix
+                    const uint32_t rbase = ka + (uint32_t)((row >> 3) * 2048 + (row & 7) * 128);
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const int c16 = ks * 2 + (lane >> 4); // 16-byte chunk of the row: dims [8 c16, 8 c16 + 8)
+                        const uint32_t coff = (uint32_t)((c16 >> 3) * 1024 + (((c16 & 7) ^ (row & 7)) << 4));
+#pragma unroll
+                        for (int mb = 0; mb < 8; ++mb) {
                             unsigned a0, a1, a2, a3;
                             asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
-                                         : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3) : "r"(addr));
+                                         : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3) : "r"(rbase + coff + (uint32_t)(mb * 4096)));
                             asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
-                                         : "+f"(c0), "+f"(c1), "+f"(c2), "+f"(c3)
+                                         : "+f"(c[mb][0]), "+f"(c[mb][1]), "+f"(c[mb][2]), "+f"(c[mb][3])
                                          : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(breg[ks][0]), "r"(breg[ks][1]));
                         }
-                        // this lane holds, for rows lane / 4 and lane / 4 + 8 of the block, both columns of head lane % 4
-                        sh.lin[lb][mb * 16 + (lane >> 2)][lane & 3] = (c0 + c1) * c_lin;
-                        sh.lin[lb][mb * 16 + (lane >> 2) + 8][lane & 3] = (c2 + c3) * c_lin;
+                    }
+                    // this lane holds, for rows lane / 4 and lane / 4 + 8 of each block, both columns of head lane % 4
+#pragma unroll
+                    for (int mb = 0; mb < 8; ++mb) {
+                        sh.lin[lb][mb * 16 + (lane >> 2)][lane & 3] = (c[mb][0] + c[mb][1]) * c_lin;
+                        sh.lin[lb][mb * 16 + (lane >> 2) + 8][lane & 3] = (c[mb][2] + c[mb][3]) * c_lin;
                     }
                     __syncwarp();
                     if (lane == 0) { mbar_arrive(smem_u32(&sh.linfull[lb])); mbar_arrive(smem_u32(&sh.kempty[st])); }
@@ -255,18 +259,20 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_expected_tc(DevParams p, cons
                 const long long g = g_begin + gv % g_span;
                 const Segment s = decode_segment(p, prefix, tiles_lh, tpc, g, g_end, my_h);
                 const int T = s.T;
-                if (q4 == 0)
-                    for (int rb = 0; rb < kExHeads; ++rb) sh.stat[rb][li] = make_float2(-INFINITY, 0.0f);
+                if (q4 < kExHeads) sh.stat[q4][li] = make_float2(-INFINITY, 0.0f); // warpgroup rb keeps the statistics of head rb
                 asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
                 float *lg_out = p.ex_logits + ((size_t)s.uid * p.G + p.ex_g0) * p.T_cap;
-                for (int i = 0; i < s.n && ok; ++i, ++kit) {
+                // A thread whose wait ran out keeps walking tiles and heads without touching the pipeline: the named
+                // barriers below have no time limit, so every consumer thread must reach each of them.
+                for (int i = 0; i < s.n; ++i, ++kit) {
                     const int t0 = (s.tile0 + i) * kTileTokens;
-                    const int st = kit % NS;
-                    ok = mbar_wait(smem_u32(&sh.kfull[st]), (uint32_t)((kit / NS) & 1), abort_flag);
-                    if (!ok) break;
-                    // this thread's quarter of its token's key: four 16-byte chunks, un-swizzled by the row number
+                    const int st = kit % NS, lb = kit & 1;
                     unsigned long long kf[16];
-                    {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) kf[j] = 0ull;
+                    if (ok) ok = mbar_wait(smem_u32(&sh.kfull[st]), (uint32_t)((kit / NS) & 1), abort_flag);
+                    if (ok) {
+                        // this thread's quarter of its token's key: four 16-byte chunks, un-swizzled by the row number
                         const unsigned char *row = Ks + (size_t)st * kTileBytes + (li >> 3) * 2048 + (q4 >> 1) * 1024 + (li & 7) * 128;
 #pragma unroll
                         for (int cch = 0; cch < 4; ++cch) {
@@ -278,38 +284,37 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_expected_tc(DevParams p, cons
                         }
                     }
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&sh.kempty[st]));
-                    const int lb = kit & 1;
-                    if (q4 == 0) { // the mean terms of this tile (warp 2)
-                        ok = mbar_wait(smem_u32(&sh.linfull[lb]), (uint32_t)((kit >> 1) & 1), abort_flag);
-                        if (!ok) break;
-                    }
-                    for (int rb = 0; rb < n_rb && ok; ++rb) {
+                    if (ok && lane == 0) mbar_arrive(smem_u32(&sh.kempty[st]));
+                    // the mean terms of this tile (warp 2); warpgroup rb reads those of head rb
+                    if (ok && q4 < n_rb) ok = mbar_wait(smem_u32(&sh.linfull[lb]), (uint32_t)((kit >> 1) & 1), abort_flag);
+                    for (int rb = 0; rb < n_rb; ++rb) {
                         const int slot = rb;
-                        const uint32_t use_parity = (uint32_t)(kit & 1);
-                        ok = mbar_wait(smem_u32(&sh.tfull[slot]), use_parity, abort_flag);
-                        if (!ok) break;
-                        tc_fence_after();
-                        const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * 128 + q4 * 32);
-                        uint32_t d[32];
-                        tc_ld32_issue(taddr, d);
-                        tc_ld_wait(d);
-                        unsigned long long aq2 = 0ull;
+                        float val = 0.0f;
+                        if (ok) ok = mbar_wait(smem_u32(&sh.tfull[slot]), (uint32_t)(kit & 1), abort_flag);
+                        ok = __all_sync(0xffffffffu, ok) != 0; // one answer per warp: the accumulator loads below are warp-wide
+                        if (ok) {
+                            tc_fence_after();
+                            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * 128 + q4 * 32);
+                            uint32_t d[32];
+                            tc_ld32_issue(taddr, d);
+                            tc_ld_wait(d);
+                            unsigned long long aq2 = 0ull;
 #pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            aq2 = fma_f32x2(pack_f32x2(__uint_as_float(d[2 * j]), __uint_as_float(d[2 * j + 1])), kf[j], aq2);
-                        float val = sum_f32x2(aq2) * c_quad; // this quarter's part of the quadratic term, in log2 units
-                        // The four quarters of the columns meet here: warpgroups 1-3 leave their parts in shared memory,
-                        // warpgroup 0 adds them.  The buffer belongs to the slot, and warpgroup 0 releases the slot only
-                        // after reading it, so the next use of the slot cannot overwrite it early.
-                        const uint32_t pbar = smem_u32(&sh.pfull[slot]);
-                        if (q4 != 0) {
-                            sh.pacc[slot][q4 - 1][li] = val;
+                            for (int j = 0; j < 16; ++j)
+                                aq2 = fma_f32x2(pack_f32x2(__uint_as_float(d[2 * j]), __uint_as_float(d[2 * j + 1])), kf[j], aq2);
+                            val = sum_f32x2(aq2) * c_quad; // this quarter's part of the quadratic term, in log2 units
+                        }
+                        // The four quarters of the columns meet in warpgroup rb (the heads take turns, so that the extra work is
+                        // spread): the others leave their parts in the slot's buffer and arrive at the slot's named barrier, warpgroup
+                        // rb waits there, adds and stores.  It releases the slot only after reading the buffer, so the next use
+                        // of the slot cannot overwrite it early.
+                        if (q4 != rb) {
+                            sh.pacc[slot][q4 < rb ? q4 : q4 - 1][li] = val;
                             tc_fence_before();
-                            __syncwarp();
-                            if (lane == 0) { mbar_arrive(pbar); mbar_arrive(smem_u32(&sh.tempty[slot])); }
+                            asm volatile("bar.arrive %0, %1;" ::"r"(2 + slot), "n"(kConsumerThreads) : "memory");
+                            if (ok && lane == 0) mbar_arrive(smem_u32(&sh.tempty[slot]));
                         } else {
-                            ok = mbar_wait(pbar, use_parity, abort_flag);
+                            asm volatile("bar.sync %0, %1;" ::"r"(2 + slot), "n"(kConsumerThreads) : "memory");
                             if (ok) {
                                 val += (sh.pacc[slot][0][li] + sh.pacc[slot][1][li]) + (sh.pacc[slot][2][li] + sh.lin[lb][li][rb]);
                                 const int t = t0 + li;
@@ -321,27 +326,20 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_expected_tc(DevParams p, cons
                                 }
                                 tc_fence_before();
                                 __syncwarp();
-                                if (lane == 0) mbar_arrive(smem_u32(&sh.tempty[slot]));
+                                if (lane == 0) { mbar_arrive(smem_u32(&sh.tempty[slot])); mbar_arrive(smem_u32(&sh.linempty[lb])); }
                             }
                         }
                     }
-                    if (q4 == 0 && ok) { // the mean-term buffer may be refilled
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(smem_u32(&sh.linempty[lb]));
-                    }
                 }
-                // fold warpgroup 0's statistics in a fixed order and store this block's part of the unit
-                if (q4 == 0) {
+                // fold each head's statistics (warpgroup rb, its four warps in a fixed order) and store this block's part of the unit
+                {
+                    float mm = sh.stat[q4][li].x, zz = sh.stat[q4][li].y;
 #pragma unroll
-                    for (int rb = 0; rb < kExHeads; ++rb) {
-                        float mm = sh.stat[rb][li].x, zz = sh.stat[rb][li].y;
-#pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) {
-                            const float m2 = __shfl_xor_sync(0xffffffffu, mm, o), z2 = __shfl_xor_sync(0xffffffffu, zz, o);
-                            lse_merge(mm, zz, m2, z2);
-                        }
-                        if (lane == 0) sh.red[quad][rb] = make_float2(mm, zz);
+                    for (int o = 16; o > 0; o >>= 1) {
+                        const float m2 = __shfl_xor_sync(0xffffffffu, mm, o), z2 = __shfl_xor_sync(0xffffffffu, zz, o);
+                        lse_merge(mm, zz, m2, z2);
                     }
+                    if (lane == 0) sh.red[quad][q4] = make_float2(mm, zz);
                 }
                 asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
                 if (warp == 4 && lane < n_rb && ok) {
