@@ -273,10 +273,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_expected_tc(DevParams p, cons
                     if (ok) ok = mbar_wait(smem_u32(&sh.kfull[st]), (uint32_t)((kit / NS) & 1), abort_flag);
                     if (ok) {
                         // this thread's quarter of its token's key: four 16-byte chunks, un-swizzled by the row number
-                        const unsigned char *row = Ks + (size_t)st * kTileBytes + (li >> 3) * 2048 + (q4 >> 1) * 1024 + (li & 7) * 128;
+                        const uint32_t row = smem_u32(Ks) + (uint32_t)(st * kTileBytes + (li >> 3) * 2048 + (q4 >> 1) * 1024 + (li & 7) * 128);
 #pragma unroll
                         for (int cch = 0; cch < 4; ++cch) {
-                            const uint4 v = *reinterpret_cast<const uint4 *>(row + ((((q4 & 1) * 4 + cch) ^ (li & 7)) << 4));
+                            uint4 v;
+                            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                                         : "r"(row + (uint32_t)((((q4 & 1) * 4 + cch) ^ (li & 7)) << 4)));
                             kf[4 * cch] = pack_f32x2(bf16_lo(v.x), bf16_hi(v.x));
                             kf[4 * cch + 1] = pack_f32x2(bf16_lo(v.y), bf16_hi(v.y));
                             kf[4 * cch + 2] = pack_f32x2(bf16_lo(v.z), bf16_hi(v.z));
