@@ -346,13 +346,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
                             if (ok) {
                                 acc += pa[li];
                                 const int t = t0 + li;
+                                // the slot is released before the usage goes to global memory: an arrive (a release) issued
+                                // after the store would wait until the store has been performed
+                                tc_fence_before();
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(smem_u32(&sh.tempty[last_slot]));
                                 if (t < T) {
                                     const int ninv = p.causal ? p.G * max(0, t - (T - p.W)) : 0;
                                     p.scores[(size_t)s.uid * p.T_cap + t] = (acc + (float)ninv * pmax) * (1.0f / (float)p.rows);
                                 }
-                                tc_fence_before();
-                                __syncwarp();
-                                if (lane == 0) mbar_arrive(smem_u32(&sh.tempty[last_slot]));
                             }
                         }
                         if (bit) ++pc1; else ++pc0;
