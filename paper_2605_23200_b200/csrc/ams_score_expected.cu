@@ -364,6 +364,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_expected_tc(DevParams p, cons
 }
 
 constexpr int kFinThreads = 256; // 16 token rows x 16 lanes of 16 bytes
+constexpr int kFinSlice = 2048;  // tokens per block: long enough to pay for merging the unit's statistics first
 
 // score_t = (mean over the group's heads of 2^(l_{r,t} - b_r) + eps) * |v_t|, b_r = M_r + log2 Z_r merged from the
 // parts the blocks of the first kernel left (an unused part is all zero).
@@ -375,16 +376,23 @@ __global__ void __launch_bounds__(kFinThreads) k_expected_final(DevParams p)
     const int h = uid % p.H, b = (uid / p.H) % p.B, l = uid / (p.H * p.B);
     const int T = p.seq_lens[b];
     if (T <= p.Tk || T > p.T_cap) return;
-    const int t_begin = slice * p.slice_len;
+    const int t_begin = slice * kFinSlice;
     if (t_begin >= T) return;
-    const int t_end = min(T, t_begin + p.slice_len);
-    if (threadIdx.x < p.G) {
+    const int t_end = min(T, t_begin + kFinSlice);
+    // warp w merges the parts of heads w, w + 8, ...: one part per lane (their loads in flight together), then a
+    // fixed tree over the lanes
+    for (int hd = threadIdx.x >> 5; hd < p.G; hd += kFinThreads / 32) {
         float mm = -INFINITY, zz = 0.0f;
-        for (int q = 0; q < p.n_slices; ++q) {
-            const float2 v = __ldcg(reinterpret_cast<const float2 *>(p.part) + ((size_t)uid * p.n_slices + q) * p.G + threadIdx.x);
-            if (v.y > 0.0f) lse_merge(mm, zz, v.x, v.y);
+        for (int q = threadIdx.x & 31; q < p.n_slices; q += 32) {
+            const float2 v = __ldcg(reinterpret_cast<const float2 *>(p.part) + ((size_t)uid * p.n_slices + q) * p.G + hd);
+            if (v.y > 0.0f) tc::lse_merge(mm, zz, v.x, v.y);
         }
-        b_s[threadIdx.x] = zz > 0.0f ? mm + log2f(zz) : INFINITY;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float m2 = __shfl_xor_sync(0xffffffffu, mm, o), z2 = __shfl_xor_sync(0xffffffffu, zz, o);
+            tc::lse_merge(mm, zz, m2, z2);
+        }
+        if ((threadIdx.x & 31) == 0) b_s[hd] = zz > 0.0f ? mm + log2f(zz) : INFINITY;
     }
     __syncthreads();
     const int lane = threadIdx.x & 15, r = threadIdx.x >> 4;
@@ -477,7 +485,7 @@ int launch_score_expected(const DevParams &p_in, LaunchCtx &ctx)
         k_expected_tc<<<tg.grid, kTcThreads, smem, ctx.s>>>(p, k_map, c_map);
         ctx.mark(kKernScore1);
     }
-    const dim3 grid(p.n_slices, (unsigned)U);
+    const dim3 grid((unsigned)((p.T_cap + kFinSlice - 1) / kFinSlice), (unsigned)U);
     if (launch_after(k_expected_final, grid, dim3(kFinThreads), 0, ctx.s, p) != cudaSuccess) return AMS_ERR_CUDA;
     ctx.mark(kKernScore2);
     return cudaGetLastError() == cudaSuccess ? AMS_OK : AMS_ERR_CUDA;

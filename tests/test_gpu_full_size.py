@@ -30,7 +30,7 @@ class _LightSnapshot:
         self.lens = cache.seq_lens.cpu().numpy().copy()
 
 
-def _sampled_units_match_the_oracle(wl, cache, comp, snap, dbg, sample, k_before, credit_zero, atol=0.0):
+def _sampled_units_match_the_oracle(wl, cache, comp, snap, dbg, sample, k_before, credit_zero, atol=0.0, v_before=None, stats=None):
     """Scores and mass of the sampled units within 1e-3 of the oracle; on the library's own scores the oracle
     must select exactly what the library selected (segments, quotas, kept positions, mass, credit)."""
     G, Tk = wl.group, wl.budget
@@ -41,6 +41,10 @@ def _sampled_units_match_the_oracle(wl, cache, comp, snap, dbg, sample, k_before
         if wl.scorer_id == inputs.SCORER_TOVA:
             q = inputs.as_u16(cache.obs_queries[l, b, h * G:(h + 1) * G])
             want = oracle.score_tova(k_l, 0, h, snap.table[b], T, q, G, wl.window, True)
+        elif wl.scorer_id == inputs.SCORER_EXPECTED:
+            mean, cov = stats
+            want = oracle.score_expected(k_l, inputs.as_u16(v_before[l:l + 1]), 0, h, snap.table[b], T,
+                                         mean[l, b, h * G:(h + 1) * G].cpu().numpy(), inputs.as_u16(cov[l, b, h * G:(h + 1) * G]), 1e-2)
         else:
             want = oracle.score_keydiff(k_l, 0, h, snap.table[b], T)
         got = dbg.scores[l, b, h, :T].cpu().numpy()
@@ -117,6 +121,10 @@ def _properties_of_every_unit(wl, cache, comp, dbg, snap, dst, k_before, v_befor
 def _run(wl, sample, atol=0.0, launches=None):
     cache = inputs.make_cache(wl, DEV)
     comp = binding.AmsCompressor(binding.config_for(wl), DEV)
+    stats = None
+    if wl.scorer_id == inputs.SCORER_EXPECTED:
+        stats = inputs.make_query_stats(cache)
+        comp.set_query_stats(stats[0], stats[1], 1e-2)
     snap = _LightSnapshot(cache)
     credit_zero = float(comp.ema_state.abs().sum()) == 0.0
     k_before = cache.k_pages.clone()
@@ -125,7 +133,7 @@ def _run(wl, sample, atol=0.0, launches=None):
     dbg = gpu_event(comp, cache, dst)
     if launches is not None:
         assert comp.last_launch_count == launches
-    _sampled_units_match_the_oracle(wl, cache, comp, snap, dbg, sample, k_before, credit_zero, atol)
+    _sampled_units_match_the_oracle(wl, cache, comp, snap, dbg, sample, k_before, credit_zero, atol, v_before, stats)
     _properties_of_every_unit(wl, cache, comp, dbg, snap, dst, k_before, v_before)
 
 
@@ -142,3 +150,8 @@ def test_config2_whole_ragged_batch_properties():
 def test_config3_one_four_layer_launch_properties():
     wl = inputs.CONFIGS[3]
     _run(wl, [(0, 0, 0), (3, 63, 7)], atol=1e-5)
+
+
+def test_expected_attention_workload_sampled_units_and_properties():
+    """The extension workload of the benchmark (geometry of configuration 1, expected-attention scorer) at its timed size."""
+    _run(inputs.CONFIGS[5], [(0, 0, 0), (17, 0, 5), (31, 0, 7)], launches=8)
