@@ -60,11 +60,12 @@ __global__ void __launch_bounds__(kTovaThreads) k_tova(DevParams p)
     __shared__ __align__(16) __nv_bfloat16 Qs[NTB > 1 ? NTB * 8 * kQPitch : 8];
     __shared__ float red[4][NTB * 8][2];
     if (PHASE == 2) wait_for_previous_kernel(); // merged statistics
-    const int uid = blockIdx.y, slice = blockIdx.x;
+    const int uid = blockIdx.y;
     const int h = uid % p.H, b = (uid / p.H) % p.B, l = uid / (p.H * p.B);
     const int T = p.seq_lens[b];
     if (T <= p.Tk || T > p.T_cap) return;
-    if (p.W > T) { if (PHASE == 1 && slice == 0 && threadIdx.x == 0) set_status(p.status, AMS_ERR_INVALID_ARG, uid, p.W, T); return; }
+    if (p.W > T) { if (PHASE == 1 && blockIdx.x == 0 && threadIdx.x == 0) set_status(p.status, AMS_ERR_INVALID_ARG, uid, p.W, T); return; }
+    const int slice = blockIdx.x;
     const int t_begin = slice * p.slice_len;
     if (t_begin >= T) return;
     const int t_end = min(T, t_begin + p.slice_len);
@@ -255,20 +256,25 @@ __global__ void __launch_bounds__(256) k_tova_usage_from_logits(DevParams p)
     const float *fin = p.fin + (size_t)uid * (p.rows_pad + 8);
     if (threadIdx.x <= RP) bs[threadIdx.x] = fin[threadIdx.x]; // b_r of the rows, then the window maximum
     __syncthreads();
-    const int t = blockIdx.y * 256 + threadIdx.x;
-    if (t >= T) return;
-    const float4 *x = reinterpret_cast<const float4 *>(p.logits + ((size_t)uid * p.T_cap + t) * RP);
-    float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    // a block takes several tiles of 256 tokens (up to eight at large capacities), so that the statistics above are
+    // fetched once per 2048 tokens and a sequence far below the capacity costs few idle blocks
+    const int tiles = ((p.T_cap + 255) / 256 + gridDim.y - 1) / gridDim.y;
+    for (int tile = 0; tile < tiles; ++tile) {
+        const int t = (blockIdx.y * tiles + tile) * 256 + threadIdx.x;
+        if (t >= T) return;
+        const float4 *x = reinterpret_cast<const float4 *>(p.logits + ((size_t)uid * p.T_cap + t) * RP);
+        float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
-    for (int q = 0; q < RP / 4; ++q) {
-        const float4 v = __ldcs(x + q);
-        acc[0] += ex2(v.x - bs[4 * q]);
-        acc[1] += ex2(v.y - bs[4 * q + 1]);
-        acc[2] += ex2(v.z - bs[4 * q + 2]);
-        acc[3] += ex2(v.w - bs[4 * q + 3]);
+        for (int q = 0; q < RP / 4; ++q) {
+            const float4 v = __ldcs(x + q);
+            acc[0] += ex2(v.x - bs[4 * q]);
+            acc[1] += ex2(v.y - bs[4 * q + 1]);
+            acc[2] += ex2(v.z - bs[4 * q + 2]);
+            acc[3] += ex2(v.w - bs[4 * q + 3]);
+        }
+        const int ninv = p.causal ? p.G * max(0, t - (T - p.W)) : 0;
+        p.scores[(size_t)uid * p.T_cap + t] = ((acc[0] + acc[1]) + (acc[2] + acc[3]) + (float)ninv * bs[RP]) * (1.0f / (float)p.rows);
     }
-    const int ninv = p.causal ? p.G * max(0, t - (T - p.W)) : 0;
-    p.scores[(size_t)uid * p.T_cap + t] = ((acc[0] + acc[1]) + (acc[2] + acc[3]) + (float)ninv * bs[RP]) * (1.0f / (float)p.rows);
 }
 
 // ---------------------------------------------------------------------------- KeyDiff
@@ -404,7 +410,8 @@ void launch_tova_ntb(const DevParams &p, LaunchCtx &ctx)
     launch_after(k_tova_combine, dim3((unsigned)(p.L * p.B * p.H)), dim3(128), 0, ctx.s, p);
     ctx.mark(kKernScoreCombine);
     if (NTB <= 2 && p.logits && p.rows_pad == NTB * 8) {
-        const dim3 g2(p.L * p.B * p.H, (p.T_cap + 255) / 256);
+        const int n256 = (p.T_cap + 255) / 256, per = n256 >= 128 ? 8 : (n256 >= 32 ? n256 / 16 : 1); // tiles per block
+        const dim3 g2(p.L * p.B * p.H, (n256 + per - 1) / per);
         launch_after(k_tova_usage_from_logits<NTB * 8>, g2, dim3(256), 0, ctx.s, p);
     } else {
         launch_after(k_tova<NTB, 2>, grid, dim3(kTovaThreads), 0, ctx.s, p);
