@@ -289,6 +289,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_expected_tc(DevParams p, cons
                     if (ok && lane == 0) mbar_arrive(smem_u32(&sh.kempty[st]));
                     // the mean terms of this tile (warp 2); warpgroup rb reads those of head rb
                     if (ok && q4 < n_rb) ok = mbar_wait(smem_u32(&sh.linfull[lb]), (uint32_t)((kit >> 1) & 1), abort_flag);
+                    float my_part = 0.0f; // this warpgroup's quarter of its own head (head q4), until the others' parts are in
                     for (int rb = 0; rb < n_rb; ++rb) {
                         const int slot = rb;
                         float val = 0.0f;
@@ -308,27 +309,32 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_expected_tc(DevParams p, cons
                         }
                         // The four quarters of the columns meet in warpgroup rb (the heads take turns, so that the extra work is
                         // spread): the others leave their parts in the slot's buffer and arrive at the slot's named barrier, warpgroup
-                        // rb waits there, adds and stores.  It releases the slot only after reading the buffer, so the next use
-                        // of the slot cannot overwrite it early.
+                        // rb waits there, adds and stores, and releases the slot only after reading the buffer, so the next use of
+                        // the slot cannot overwrite it early.  It does so one head late, after delivering its part of head rb + 1:
+                        // otherwise every head would wait for the warpgroup that has just added up the one before.
                         if (q4 != rb) {
                             sh.pacc[slot][q4 < rb ? q4 : q4 - 1][li] = val;
                             tc_fence_before();
                             asm volatile("bar.arrive %0, %1;" ::"r"(2 + slot), "n"(kConsumerThreads) : "memory");
                             if (ok && lane == 0) mbar_arrive(smem_u32(&sh.tempty[slot]));
                         } else {
-                            asm volatile("bar.sync %0, %1;" ::"r"(2 + slot), "n"(kConsumerThreads) : "memory");
+                            my_part = val;
+                        }
+                        if (q4 < n_rb && (rb == q4 + 1 || (rb == q4 && rb == n_rb - 1))) {
+                            // this warpgroup's own head: slot q4
+                            asm volatile("bar.sync %0, %1;" ::"r"(2 + q4), "n"(kConsumerThreads) : "memory");
                             if (ok) {
-                                val += (sh.pacc[slot][0][li] + sh.pacc[slot][1][li]) + (sh.pacc[slot][2][li] + sh.lin[lb][li][rb]);
+                                const float lg2 = my_part + (sh.pacc[q4][0][li] + sh.pacc[q4][1][li]) + (sh.pacc[q4][2][li] + sh.lin[lb][li][q4]);
                                 const int t = t0 + li;
                                 if (t < T) {
-                                    lg_out[(size_t)rb * p.T_cap + t] = val;
-                                    const float2 mz = sh.stat[rb][li];
-                                    const float mn = fmaxf(mz.x, val);
-                                    sh.stat[rb][li] = make_float2(mn, mz.y * ex2(mz.x - mn) + ex2(val - mn));
+                                    lg_out[(size_t)q4 * p.T_cap + t] = lg2;
+                                    const float2 mz = sh.stat[q4][li];
+                                    const float mn = fmaxf(mz.x, lg2);
+                                    sh.stat[q4][li] = make_float2(mn, mz.y * ex2(mz.x - mn) + ex2(lg2 - mn));
                                 }
                                 tc_fence_before();
                                 __syncwarp();
-                                if (lane == 0) { mbar_arrive(smem_u32(&sh.tempty[slot])); mbar_arrive(smem_u32(&sh.linempty[lb])); }
+                                if (lane == 0) { mbar_arrive(smem_u32(&sh.tempty[q4])); mbar_arrive(smem_u32(&sh.linempty[lb])); }
                             }
                         }
                     }
