@@ -117,3 +117,29 @@ def test_expected_needs_room_and_statistics():
         plain.compress(cache.k_pages, cache.v_pages, cache.block_table, cache.seq_lens, None, wl.budget, wl.n_segments,
                        inputs.SCORER_EXPECTED, dst)
     assert e.value.code == binding.AMS_ERR_CAPACITY
+
+
+def test_expected_two_events_with_credit_carried():
+    """Two consecutive events with appended tokens in between (EMA on): the credit carried in compacted order, the
+    rewritten block table and fresh query statistics feed the second event."""
+    wl = _wl(n_layers=1, batch=2, seq_len_min=2000, seq_len_max=3000, budget=768, append_per_step=256, steps=2)
+    cache = inputs.make_cache(wl, DEV)
+    comp = binding.AmsCompressor(binding.config_for(wl), DEV)
+    for ev in range(2):
+        if ev:
+            inputs.append_tokens(cache, wl.append_per_step)
+        mean, cov = inputs.make_query_stats(cache)
+        comp.set_query_stats(mean, cov, EPS)
+        snap = HostSnapshot(cache)
+        credit0 = comp.ema_state.cpu().numpy()
+        assert (credit0 != 0).any() == bool(ev)
+        dst = inputs.alloc_dst_pages(cache)
+        dbg = gpu_event(comp, cache, dst)
+        got = dbg.scores.cpu().numpy()
+        units = [(0, b, h) for b in range(wl.batch) for h in range(wl.n_kv_heads)]
+        want = _oracle_scores(snap, wl, mean.cpu().numpy(), inputs.as_u16(cov), units)
+        for (l, b, h), w in want.items():
+            assert_scores_close(got[l, b, h, :int(snap.lens[b])], w, rtol=1e-3)
+        compare_event(snap, cache, comp, dbg, dst, credit0, got)
+        assert (cache.seq_lens.cpu().numpy() == wl.budget).all()
+        inputs.after_compress(cache, dst)
