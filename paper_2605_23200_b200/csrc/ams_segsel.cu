@@ -30,7 +30,6 @@ using namespace sel;
 
 namespace {
 
-constexpr int kScanThreads = 512;
 constexpr int kScanVec = 8;                 // tokens per thread and round of the scan pass
 constexpr int kListCap = 1024;              // backfill candidates kept in shared memory
 
@@ -47,21 +46,21 @@ __device__ __forceinline__ UnitId unit_of(const DevParams &p, int uid)
 // Walks the first `n` floats of a row (allocated to a multiple of 4) with float4 loads, four per thread in
 // flight: f(t, v, full) gets the position of the group's first element and, as a compile-time flag, whether
 // the whole group lies inside the row (then no per-element bound is needed).
-template <typename F>
+template <int NT, typename F>
 __device__ __forceinline__ void walk4(const float *row, int n, F f)
 {
     const int n4 = (n + 3) & ~3;
     const int tid = threadIdx.x;
-    for (int base = 0; base < n4; base += kScanThreads * 16) {
+    for (int base = 0; base < n4; base += NT * 16) {
         float4 v[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int t = base + (j * kScanThreads + tid) * 4;
+            const int t = base + (j * NT + tid) * 4;
             v[j] = t < n4 ? *reinterpret_cast<const float4 *>(row + t) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
         }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int t = base + (j * kScanThreads + tid) * 4;
+            const int t = base + (j * NT + tid) * 4;
             if (t + 3 < n) f(t, v[j], std::true_type{});
             else if (t < n) f(t, v[j], std::false_type{});
         }
@@ -69,22 +68,22 @@ __device__ __forceinline__ void walk4(const float *row, int n, F f)
 }
 
 // The same over two rows at once (usage and credit).
-template <typename F>
+template <int NT, typename F>
 __device__ __forceinline__ void walk4x2(const float *row_a, const float *row_b, int n, F f)
 {
     const int n4 = (n + 3) & ~3;
     const int tid = threadIdx.x;
-    for (int base = 0; base < n4; base += kScanThreads * 16) {
+    for (int base = 0; base < n4; base += NT * 16) {
         float4 va[4], vb[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int t = base + (j * kScanThreads + tid) * 4;
+            const int t = base + (j * NT + tid) * 4;
             va[j] = vb[j] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
             if (t < n4) { va[j] = *reinterpret_cast<const float4 *>(row_a + t); vb[j] = *reinterpret_cast<const float4 *>(row_b + t); }
         }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int t = base + (j * kScanThreads + tid) * 4;
+            const int t = base + (j * NT + tid) * 4;
             if (t + 3 < n) f(t, va[j], vb[j], std::true_type{});
             else if (t < n) f(t, va[j], vb[j], std::false_type{});
         }
@@ -112,7 +111,8 @@ __device__ __forceinline__ double block_sum_exact_f64(double v, u64 *scratch)
 
 // raw_cuts: [units][S + 1] cut positions of the mass quantiles (entry k: boundary after the token that
 // reaches k / S; T where no token before the last one does).
-__global__ void __launch_bounds__(kScanThreads) k_mass_scan(DevParams p)
+template <int NT>
+__global__ void __launch_bounds__(NT) k_mass_scan(DevParams p)
 {
     extern __shared__ __align__(16) unsigned char dyn[];
     __shared__ u64 scratch[40];
@@ -130,13 +130,13 @@ __global__ void __launch_bounds__(kScanThreads) k_mass_scan(DevParams p)
     const bool ema_on = p.beta != 1.0f;
     const double two_f = (double)(1ull << kFixBits);
     wait_for_previous_kernel(); // the usage scores
-    for (int k = tid; k <= p.S; k += kScanThreads) raw[k] = T;
+    for (int k = tid; k <= p.S; k += NT) raw[k] = T;
 
     // Rows are allocated to the capacity (a multiple of 16), so whole float4 groups may be read past the
     // sequence's end; what lies there is masked by position.
     // ---- largest Eq. 1 weight -> exponent of the fixed-point images
     float wmax = 0.0f;
-    walk4(u, T, [&](int t, float4 v, auto full) {
+    walk4<NT>(u, T, [&](int t, float4 v, auto full) {
         const float w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) if (decltype(full)::value || t + i < T) wmax = fmaxf(wmax, weight_of(w[i], p.eps));
@@ -147,7 +147,7 @@ __global__ void __launch_bounds__(kScanThreads) k_mass_scan(DevParams p)
     const double scale_w = fix_scale_of(ew);
     const float cut_w = fixed_trunc_threshold(ew); // weights below it lose their bits under the image's last one
     double sa = 0.0;
-    walk4(u, T, [&](int t, float4 v, auto full) {
+    walk4<NT>(u, T, [&](int t, float4 v, auto full) {
         const float w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i)
@@ -166,7 +166,7 @@ __global__ void __launch_bounds__(kScanThreads) k_mass_scan(DevParams p)
     if (ema_on) {
         const float oml = __fsub_rn(1.0f, p.lambda);
         float cmax = 0.0f;
-        walk4x2(u, credit, T, [&](int t, float4 v, float4 cv, auto full) {
+        walk4x2<NT>(u, credit, T, [&](int t, float4 v, float4 cv, auto full) {
             const float w[4] = {v.x, v.y, v.z, v.w};
             float c[4] = {cv.x, cv.y, cv.z, cv.w};
             float m[4];
@@ -194,7 +194,7 @@ __global__ void __launch_bounds__(kScanThreads) k_mass_scan(DevParams p)
             ec = fix_exponent(cmax);
             scale_c = fix_scale_of(ec);
             cut_c = fixed_trunc_threshold(ec);
-            walk4(credit, T, [&](int t, float4 cv, auto full) {
+            walk4<NT>(credit, T, [&](int t, float4 cv, auto full) {
                 const float c[4] = {cv.x, cv.y, cv.z, cv.w};
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
@@ -211,7 +211,7 @@ __global__ void __launch_bounds__(kScanThreads) k_mass_scan(DevParams p)
     //      before this round's block-wide scan
     const double bd = (double)p.beta, omb = __dsub_rn(1.0, (double)p.beta);
     u64 carry = 0;
-    constexpr int kRound = kScanThreads * kScanVec;
+    constexpr int kRound = NT * kScanVec;
     float4 wn[kScanVec / 4], cn[kScanVec / 4];
     auto fetch = [&](int base) {
 #pragma unroll
@@ -283,7 +283,7 @@ __global__ void __launch_bounds__(kScanThreads) k_mass_scan(DevParams p)
     //      the prefix before its first and at its last token of a round and walks its tokens only if a
     //      quantile lies between the two.
     const u64 SH = carry, S = (u64)p.S;
-    for (int k = tid + 1; k < p.S; k += kScanThreads) qthr[k] = ((u64)k * SH + S - 1) / S;
+    for (int k = tid + 1; k < p.S; k += NT) qthr[k] = ((u64)k * SH + S - 1) / S;
     __syncthreads(); // (also orders the prefix sums written above before the reads below)
     auto quantile = [&](u64 c) -> int { // number of k in [1, S) with qthr[k] <= c
         int lo = 0, hi = p.S - 1;
@@ -1001,12 +1001,19 @@ int launch_segsel(const DevParams &p, LaunchCtx &ctx)
     if (small_blocks ? !grant_dynamic_smem(k_select_compact<256>, smem_s, grant_s256) : !grant_dynamic_smem(k_select_compact<512>, smem_s, grant_s512))
         return AMS_ERR_CUDA;
     const size_t smem_a = (size_t)(p.S + 1) * 8;
+    // A unit's pass is a chain of block-wide reductions: with many units per SM, blocks of 256 threads (four per SM
+    // instead of two) overlap those chains better; with few units the wider block finishes its unit sooner.
+    const int n_sm = sm_count();
+    if (n_sm <= 0) return AMS_ERR_CUDA;
+    const bool narrow_scan = units >= 6 * n_sm;
     if (ctx.launches <= 1) {
         // nothing but the validation kernel ran before (caller-supplied scores): its effective lengths are read
         // before this kernel's first wait, so this launch is fully ordered after it
-        k_mass_scan<<<units, kScanThreads, smem_a, ctx.s>>>(p);
+        if (narrow_scan) k_mass_scan<256><<<units, 256, smem_a, ctx.s>>>(p);
+        else k_mass_scan<512><<<units, 512, smem_a, ctx.s>>>(p);
         if (cudaGetLastError() != cudaSuccess) return AMS_ERR_CUDA;
-    } else if (launch_after(k_mass_scan, dim3((unsigned)units), dim3(kScanThreads), smem_a, ctx.s, p) != cudaSuccess) {
+    } else if ((narrow_scan ? launch_after(k_mass_scan<256>, dim3((unsigned)units), dim3(256), smem_a, ctx.s, p)
+                            : launch_after(k_mass_scan<512>, dim3((unsigned)units), dim3(512), smem_a, ctx.s, p)) != cudaSuccess) {
         return AMS_ERR_CUDA;
     }
     ctx.mark(kKernSegmentSelect);
