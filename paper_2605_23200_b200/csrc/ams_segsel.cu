@@ -994,8 +994,11 @@ int launch_segsel(const DevParams &p, LaunchCtx &ctx)
     const size_t smem_q = quota_smem(p.seg_cap, p.S).total, smem_s = sel_smem(p.T_cap, p.seg_cap).total;
     // Long segments (no split, or a split length above a warp's reach) are searched by the whole block, one
     // after the other, a barrier per key bit: four smaller blocks per SM hide that latency better; otherwise
-    // twice the warps per unit shorten the warp-per-segment phase.
-    const bool small_blocks = p.l_max == 0 || p.l_max > 1024;
+    // twice the warps per unit shorten the warp-per-segment phase, unless there are many units per SM.
+    const int n_sm = sm_count();
+    if (n_sm <= 0) return AMS_ERR_CUDA;
+    const bool many_units = units >= 6 * n_sm; // several blocks per SM anyway: the smaller ones overlap their serial parts better
+    const bool small_blocks = p.l_max == 0 || p.l_max > 1024 || many_units;
     static SmemGrant grant_q, grant_s256, grant_s512;
     if (!grant_dynamic_smem(k_segments_quotas, smem_q, grant_q)) return AMS_ERR_CUDA;
     if (small_blocks ? !grant_dynamic_smem(k_select_compact<256>, smem_s, grant_s256) : !grant_dynamic_smem(k_select_compact<512>, smem_s, grant_s512))
@@ -1003,9 +1006,7 @@ int launch_segsel(const DevParams &p, LaunchCtx &ctx)
     const size_t smem_a = (size_t)(p.S + 1) * 8;
     // A unit's pass is a chain of block-wide reductions: with many units per SM, blocks of 256 threads (four per SM
     // instead of two) overlap those chains better; with few units the wider block finishes its unit sooner.
-    const int n_sm = sm_count();
-    if (n_sm <= 0) return AMS_ERR_CUDA;
-    const bool narrow_scan = units >= 6 * n_sm;
+    const bool narrow_scan = many_units;
     if (ctx.launches <= 1) {
         // nothing but the validation kernel ran before (caller-supplied scores): its effective lengths are read
         // before this kernel's first wait, so this launch is fully ordered after it
