@@ -53,6 +53,8 @@ struct DevParams {
     int slice_len, n_slices, rows_pad;
     int tc_tpc_min, tc_stages;        // tensor-core scorer: least tiles per block, K stages in shared memory
     int tc_hpb;                       // tensor-core scorer: KV heads a block takes one after the other (set by its launcher)
+    int merge_in_usage;               // narrow query blocks: the pass over the stored logits merges the slices' statistics itself
+                                      // (set by the launcher when there are too few units for a kernel of its own to pay)
     float *logits;                    // narrow query blocks (rows_pad <= 16): scaled logits [units][T_cap][rows_pad], or null
     // expected-attention scorer
     const float *q_mean;              // [L][B][H*G][128] mean of the future queries per query head

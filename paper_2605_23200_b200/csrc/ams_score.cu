@@ -247,15 +247,47 @@ __global__ void __launch_bounds__(128) k_tova_combine(DevParams p)
 template <int RP>
 __global__ void __launch_bounds__(256) k_tova_usage_from_logits(DevParams p)
 {
-    __shared__ float bs[RP + 1];
-    wait_for_previous_kernel(); // merged statistics (and, through that kernel, the logits)
+    __shared__ float bs[RP + 1], zinv[RP];
+    wait_for_previous_kernel(); // the slices' statistics and the logits
     const int uid = blockIdx.x;
     const int b = (uid / p.H) % p.B;
     const int T = p.seq_lens[b];
     if (T <= p.Tk || T > p.T_cap || p.W > T) return;
-    const float *fin = p.fin + (size_t)uid * (p.rows_pad + 8);
-    if (threadIdx.x <= RP) bs[threadIdx.x] = fin[threadIdx.x]; // b_r of the rows, then the window maximum
-    __syncthreads();
+    if (!p.merge_in_usage) {
+        const float *fin = p.fin + (size_t)uid * (p.rows_pad + 8);
+        if (threadIdx.x <= RP) bs[threadIdx.x] = fin[threadIdx.x]; // b_r of the rows, then the window maximum
+        __syncthreads();
+    } else {
+        // With few units (a launch-bound event) every block merges the slices' (max, sum) of its unit itself (a warp per
+        // row, a slice per lane, then a fixed tree over the lanes: the same result in every block): b_r = M_r + log2 Z_r,
+        // and the window maximum 1 / min_r Z_r.  With many units a kernel of its own does it once per unit.
+        const int ns = (T + p.slice_len - 1) / p.slice_len, lane = threadIdx.x & 31;
+        for (int r = threadIdx.x >> 5; r < RP; r += 8) {
+            float m = -INFINITY, z = 0.0f;
+            for (int sl = lane; sl < ns; sl += 32) {
+                const float2 v = __ldcg(reinterpret_cast<const float2 *>(p.part) + ((size_t)uid * p.n_slices + sl) * RP + r);
+                lse_merge(m, z, v.x, v.y);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float m2 = __shfl_xor_sync(0xffffffffu, m, o), z2 = __shfl_xor_sync(0xffffffffu, z, o);
+                lse_merge(m, z, m2, z2);
+            }
+            if (lane == 0) {
+                const bool live = r < p.rows && z > 0.0f;
+                bs[r] = live ? m + log2f(z) : INFINITY; // padding rows contribute nothing
+                zinv[r] = live ? 1.0f / z : 0.0f;
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            float best = 0.0f;
+#pragma unroll
+            for (int r = 0; r < RP; ++r) best = fmaxf(best, zinv[r]);
+            bs[RP] = best;
+        }
+        __syncthreads();
+    }
     // a block takes several tiles of 256 tokens (up to eight at large capacities), so that the statistics above are
     // fetched once per 2048 tokens and a sequence far below the capacity costs few idle blocks
     const int tiles = ((p.T_cap + 255) / 256 + gridDim.y - 1) / gridDim.y;
@@ -402,14 +434,19 @@ __global__ void __launch_bounds__(kKdThreads) k_keydiff_score(DevParams p)
 }
 
 template <int NTB>
-void launch_tova_ntb(const DevParams &p, LaunchCtx &ctx)
+void launch_tova_ntb(const DevParams &p_in, LaunchCtx &ctx)
 {
+    DevParams p = p_in;
     const dim3 grid(p.n_slices, p.L * p.B * p.H);
     k_tova<NTB, 1><<<grid, kTovaThreads, 0, ctx.s>>>(p);
     ctx.mark(kKernScore1);
-    launch_after(k_tova_combine, dim3((unsigned)(p.L * p.B * p.H)), dim3(128), 0, ctx.s, p);
-    ctx.mark(kKernScoreCombine);
-    if (NTB <= 2 && p.logits && p.rows_pad == NTB * 8) {
+    const bool from_logits = NTB <= 2 && p.logits && p.rows_pad == NTB * 8;
+    p.merge_in_usage = from_logits && p.L * p.B * p.H <= 2 * sm_count();
+    if (!p.merge_in_usage) {
+        launch_after(k_tova_combine, dim3((unsigned)(p.L * p.B * p.H)), dim3(128), 0, ctx.s, p);
+        ctx.mark(kKernScoreCombine);
+    }
+    if (from_logits) {
         const int n256 = (p.T_cap + 255) / 256, per = n256 >= 128 ? 8 : (n256 >= 32 ? n256 / 16 : 1); // tiles per block
         const dim3 g2(p.L * p.B * p.H, (n256 + per - 1) / per);
         launch_after(k_tova_usage_from_logits<NTB * 8>, g2, dim3(256), 0, ctx.s, p);
