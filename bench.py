@@ -76,8 +76,8 @@ NCU_TRAFFIC_BYTES: dict = {
     "cfg3_qwen3_8b_L36_B64_T32768_k2048_keydiff": {"score_phase1": 4 * (4_295_511_552 + 7_466_752),
                                                    "score_phase2": 4 * (4_296_070_144 + 16_274_688)},
     # four-layer capture x 8 (profiles/expected_attention_cfg5_4layers_ncu_full.md)
-    "cfg5_llama8b_L32_T16384_k2048_expected": {"score_phase1": 8 * (138_550_784 + 6_984_960),
-                                               "score_phase2": 8 * (142_663_680 + 4_107_264)},
+    "cfg5_llama8b_L32_T16384_k2048_expected": {"score_phase1": 8 * (138_548_480 + 7_237_888),
+                                               "score_phase2": 8 * (142_662_912 + 4_347_392)},
 }
 
 
