@@ -257,38 +257,45 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
                         const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * 128 + half * 64);
                         // chunks of 16 columns, the load of the next chunk in flight while this one is worked on
                         uint32_t buf[2][16];
-                        tc_ld16_issue(taddr, buf[0]);
-                        tc_ld16_wait(buf[0]);
+                        if (PHASE == 2) {
+                            tc_ld16_issue(taddr, buf[0]);
+                            tc_ld16_wait(buf[0]);
+                        }
                         if (PHASE == 1) {
+                            // 32 columns at a time: one running-maximum update (one rescaling exponential) per 32 logits, and
+                            // the maximum tree of one half can overlap the exponentials of the other
                             const int lv = min(lastv[rb], T - 1);
                             float mr = m[rb], zr = z[rb];
+                            uint32_t d[32];
+                            tc_ld32_issue(taddr, d);
 #pragma unroll
-                            for (int ch = 0; ch < 4; ++ch) {
-                                uint32_t (&cur)[16] = buf[ch & 1];
-                                if (ch < 3) tc_ld16_issue(taddr + (ch + 1) * 16, buf[(ch + 1) & 1]);
-                                const int tc0 = t0 + half * 64 + ch * 16;
+                            for (int ch = 0; ch < 2; ++ch) {
+                                tc_ld_wait(d);
+                                float v[32];
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(d[j]);
+                                if (ch == 0) tc_ld32_issue(taddr + 32, d);
+                                const int tc0 = t0 + half * 64 + ch * 32;
                                 if (tc0 <= lv) {
-                                    float v[16];
+                                    if (tc0 + 31 > lv) {
 #pragma unroll
-                                    for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(cur[j]);
-                                    if (tc0 + 15 > lv) {
-#pragma unroll
-                                        for (int j = 0; j < 16; ++j) if (tc0 + j > lv) v[j] = -INFINITY;
+                                        for (int j = 0; j < 32; ++j) if (tc0 + j > lv) v[j] = -INFINITY;
                                     }
-                                    // tree of three-input maxima instead of a chain of 15
-                                    float a5[5];
+                                    // tree of three-input maxima
+                                    float a[11];
 #pragma unroll
-                                    for (int j = 0; j < 5; ++j) a5[j] = max3(v[j], v[j + 5], v[j + 10]);
-                                    const float cm = fmaxf(max3(a5[0], a5[1], a5[2]), max3(a5[3], a5[4], v[15]));
+                                    for (int j = 0; j < 10; ++j) a[j] = max3(v[3 * j], v[3 * j + 1], v[3 * j + 2]);
+                                    a[10] = fmaxf(v[30], v[31]);
+                                    const float b0 = max3(a[0], a[1], a[2]), b1 = max3(a[3], a[4], a[5]), b2 = max3(a[6], a[7], a[8]);
+                                    const float cm = fmaxf(max3(b0, b1, b2), fmaxf(a[9], a[10]));
                                     const float mn = fmaxf(mr, cm * c);
                                     zr *= ex2(mr - mn);
                                     mr = mn;
                                     float zs[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
-                                    for (int j = 0; j < 16; ++j) zs[j & 3] += ex2(fmaf(v[j], c, -mn));
+                                    for (int j = 0; j < 32; ++j) zs[j & 3] += ex2(fmaf(v[j], c, -mn));
                                     zr += (zs[0] + zs[1]) + (zs[2] + zs[3]);
                                 }
-                                if (ch < 3) tc_ld16_wait(buf[(ch + 1) & 1]);
                             }
                             m[rb] = mr; z[rb] = zr;
                         } else {
