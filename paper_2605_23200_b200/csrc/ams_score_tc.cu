@@ -255,12 +255,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
                         if (!ok) break;
                         tc_fence_after();
                         const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * 128 + half * 64);
-                        // chunks of 16 columns, the load of the next chunk in flight while this one is worked on
-                        uint32_t buf[2][16];
-                        if (PHASE == 2) {
-                            tc_ld16_issue(taddr, buf[0]);
-                            tc_ld16_wait(buf[0]);
-                        }
                         if (PHASE == 1) {
                             // 32 columns at a time: one running-maximum update (one rescaling exponential) per 32 logits, and
                             // the maximum tree of one half can overlap the exponentials of the other
@@ -303,29 +297,30 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tova_tc(DevParams p, const __
                             const bool plain = !p.causal || t0 + kTileTokens - 1 <= T - p.W;
                             const float4 *fr4 = reinterpret_cast<const float4 *>(fs + rb * 128 + half * 64);
                             float ac[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                            uint32_t d[32];
+                            tc_ld32_issue(taddr, d);
 #pragma unroll
-                            for (int ch = 0; ch < 4; ++ch) {
-                                uint32_t (&cur)[16] = buf[ch & 1];
-                                if (ch < 3) tc_ld16_issue(taddr + (ch + 1) * 16, buf[(ch + 1) & 1]);
+                            for (int ch = 0; ch < 2; ++ch) { // 32 columns (query rows) at a time
+                                tc_ld_wait(d);
                                 if (plain) {
 #pragma unroll
-                                    for (int j4 = 0; j4 < 4; ++j4) {
-                                        const float4 f = fr4[ch * 4 + j4];
-                                        ac[0] += ex2(fmaf(__uint_as_float(cur[4 * j4]), c, -f.x));
-                                        ac[1] += ex2(fmaf(__uint_as_float(cur[4 * j4 + 1]), c, -f.y));
-                                        ac[2] += ex2(fmaf(__uint_as_float(cur[4 * j4 + 2]), c, -f.z));
-                                        ac[3] += ex2(fmaf(__uint_as_float(cur[4 * j4 + 3]), c, -f.w));
+                                    for (int j4 = 0; j4 < 8; ++j4) {
+                                        const float4 f = fr4[ch * 8 + j4];
+                                        ac[0] += ex2(fmaf(__uint_as_float(d[4 * j4]), c, -f.x));
+                                        ac[1] += ex2(fmaf(__uint_as_float(d[4 * j4 + 1]), c, -f.y));
+                                        ac[2] += ex2(fmaf(__uint_as_float(d[4 * j4 + 2]), c, -f.z));
+                                        ac[3] += ex2(fmaf(__uint_as_float(d[4 * j4 + 3]), c, -f.w));
                                     }
                                 } else {
-                                    const int rbase = rb * 128 + half * 64 + ch * 16;
+                                    const int rbase = rb * 128 + half * 64 + ch * 32;
 #pragma unroll
-                                    for (int j = 0; j < 16; ++j) {
+                                    for (int j = 0; j < 32; ++j) {
                                         const int r = rbase + j;
                                         const bool seen = t <= T - p.W + (r % p.W);
-                                        ac[j & 3] += seen ? ex2(fmaf(__uint_as_float(cur[j]), c, -fs[r])) : 0.0f;
+                                        ac[j & 3] += seen ? ex2(fmaf(__uint_as_float(d[j]), c, -fs[r])) : 0.0f;
                                     }
                                 }
-                                if (ch < 3) tc_ld16_wait(buf[(ch + 1) & 1]);
+                                if (ch == 0) tc_ld32_issue(taddr + 32, d);
                             }
                             acc += (ac[0] + ac[1]) + (ac[2] + ac[3]);
                         }
