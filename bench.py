@@ -66,18 +66,18 @@ def _peaks():
 NCU_TRAFFIC_BYTES: dict = {
     # two-layer capture (profiles/tc_scorer_cfg4_2layers_ncu_full.md) x 40: the 80-layer launch holds 50 GB, too much to
     # capture under full counters; units are independent and each is read once per pass, so traffic grows with the layers
-    "cfg4_llama70b_L80_T131072_k8192_w64": {"score_phase1": 40 * (540_759_808 + 5_955_840),
-                                            "score_phase2": 40 * (542_750_976 + 10_740_224)},
+    "cfg4_llama70b_L80_T131072_k8192_w64": {"score_phase1": 40 * (540_616_448 + 6_414_080),
+                                            "score_phase2": 40 * (542_741_760 + 11_199_488)},
     # captured at the timed size (profiles/tc_scorer_cfg1_32layers_ncu_full.md, profiles/gather_cfg1_cfg2_ncu_full.md)
-    "cfg1_llama8b_L32_T16384_k2048_w32": {"score_phase1": 1_089_487_616 + 13_931_520,
-                                          "score_phase2": 1_090_557_184 + 19_021_568,
+    "cfg1_llama8b_L32_T16384_k2048_w32": {"score_phase1": 1_089_513_472 + 14_958_336,
+                                          "score_phase2": 1_090_619_136 + 20_133_632,
                                           "gather": 270_614_528 + 219_303_168},
     # one-layer capture x 4 resident layers (profiles/keydiff_cfg3_1layer_ncu_full.md)
     "cfg3_qwen3_8b_L36_B64_T32768_k2048_keydiff": {"score_phase1": 4 * (4_295_511_552 + 7_466_752),
                                                    "score_phase2": 4 * (4_296_070_144 + 16_274_688)},
     # four-layer capture x 8 (profiles/expected_attention_cfg5_4layers_ncu_full.md)
-    "cfg5_llama8b_L32_T16384_k2048_expected": {"score_phase1": 8 * (138_548_480 + 7_237_888),
-                                               "score_phase2": 8 * (142_662_912 + 4_347_392)},
+    "cfg5_llama8b_L32_T16384_k2048_expected": {"score_phase1": 8 * (138_547_456 + 6_842_624),
+                                               "score_phase2": 8 * (142_662_656 + 4_295_936)},
 }
 
 
