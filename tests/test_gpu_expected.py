@@ -143,3 +143,11 @@ def test_expected_two_events_with_credit_carried():
         compare_event(snap, cache, comp, dbg, dst, credit0, got)
         assert (cache.seq_lens.cpu().numpy() == wl.budget).all()
         inputs.after_compress(cache, dst)
+
+
+def test_expected_longest_sequence():
+    """131072 tokens (the capacity limit): 1024 tiles per unit, shared by some thirty blocks whose statistics are merged."""
+    wl = _wl(n_layers=1, batch=1, n_kv_heads=1, n_q_heads=2, seq_len_min=131072, seq_len_max=131072, budget=4096,
+             n_segments=32, l_max=8192)
+    cache, comp, snap, credit0, dst, dbg, got, units = _run(wl)
+    compare_event(snap, cache, comp, dbg, dst, credit0, got)
